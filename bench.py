@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the module-wise outer synchronisation (DiPaCo, Algorithm 1, outer loop).
+
+One step = one full synchronisation of the 16x16-module, 256-path, 150M-parameters-per-path
+workload (bf16 path copies, fp32 module state): outer gradients, segmented reduction over the
+paths sharing each module, Nesterov update, write-back into every path.  Prints one JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "outer_sync_path_params_per_s"
+UNIT = "path-params/s"
+CPU_SAMPLE_NUMEL = 4_000_000      # parameters per level in the CPU-baseline sample
+REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the reference arm
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="grid16x16")
+    ap.add_argument("--level-numel", type=int, default=0,
+                    help="override the parameters per level (smaller runs for profiling)")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "vector", "scalar"])
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--units", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-chunked", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of one GPU while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return world, rank, local
+
+
+def aggregate(ms_local, units_local, world, backend_device):
+    """(max ms over ranks, total units over ranks); a no-op without torch.distributed."""
+    import torch
+    import torch.distributed as dist
+    if world <= 1 or not dist.is_initialized():
+        return ms_local, units_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=backend_device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier(world):
+    import torch.distributed as dist
+    if world > 1 and dist.is_initialized():
+        dist.barrier()
+
+
+def workload_config(args):
+    from paper_2403_10616_b200 import synth
+    cfg = synth.CONFIGS[args.workload]
+    if args.level_numel:
+        cfg = cfg.scaled(tuple(args.level_numel for _ in cfg.level_numel),
+                         name="%s-n%d" % (cfg.name, args.level_numel))
+    return cfg
+
+
+def time_steps(fn, steps, world):
+    """K calls of fn between barrier + synchronize; returns (ms per step over the whole region,
+    mean per-call ms from per-step event pairs)."""
+    import torch
+    stream = torch.cuda.current_stream()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    barrier(world)
+    torch.cuda.synchronize()
+    for k in range(steps):
+        starts[k].record(stream)
+        fn()
+        ends[k].record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    total = starts[0].elapsed_time(ends[-1])
+    per_call = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    return total / steps, sum(per_call) / steps
+
+
+def cpu_baseline_from_device(problem, sample_numel):
+    """Oracle on a slab of the same workload: the first `sample_numel` parameters of every module
+    and of every path's slot, copied back from the device."""
+    import torch
+    import oracle
+    from paper_2403_10616_b200 import synth
+    cfg = problem.cfg
+    n = [min(sample_numel, x) for x in cfg.level_numel]
+    small = cfg.scaled(n)
+    mod_off = problem.module_offsets()
+    lvl_off = problem.level_offsets()
+    theta_parts, mom_parts = [], []
+    for l, k in enumerate(cfg.modules_per_level):
+        for e in range(k):
+            src = int(mod_off[l]) + e * cfg.level_numel[l]
+            theta_parts.append(problem.theta[src:src + n[l]])
+            mom_parts.append(problem.momentum[src:src + n[l]])
+    theta = torch.cat(theta_parts).cpu().numpy()
+    momentum = torch.cat(mom_parts).cpu().numpy()
+    paths = []
+    for p in problem.paths:
+        row = torch.cat([p[int(lvl_off[l]):int(lvl_off[l]) + n[l]] for l in range(cfg.num_levels)])
+        row = row.cpu()
+        if row.dtype == torch.bfloat16:
+            paths.append(row.view(torch.int16).numpy().view(np.uint16))
+        else:
+            paths.append(row.numpy())
+    threads = oracle.max_threads()
+    dtype = oracle.BF16 if cfg.path_dtype == "bf16" else oracle.F32
+    t0 = time.perf_counter()
+    oracle.outer_sync(small.modules_per_level, small.level_numel, problem.table, theta, momentum,
+                      paths, dtype, float(np.float32(cfg.outer_lr)),
+                      float(np.float32(cfg.outer_momentum)), problem.weights, problem.reported,
+                      threads)
+    dt = time.perf_counter() - t0
+    return {"value": small.path_params / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "seconds": dt,
+            "sample": "one call on the first %s parameters of every level of all %d paths (%d "
+                      "path-params), inputs copied back from the device" %
+                      ("/".join(str(x) for x in n), cfg.num_paths, small.path_params)}
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the workload per step."""
+    world, rank, _ = dist_setup(args)
+    if rank != 0:
+        return
+    import oracle
+    from paper_2403_10616_b200 import synth
+    cfg = workload_config(args)
+    n = [min(REF_SAMPLE_NUMEL, x) for x in cfg.level_numel]
+    small = cfg.scaled(n)
+    pr = synth.make_problem(small, "cpu")
+    theta = pr.theta.numpy()
+    momentum = pr.momentum.numpy()
+    import torch
+    if small.path_dtype == "bf16":
+        paths = [p.view(torch.int16).numpy().view(np.uint16) for p in pr.paths]
+    else:
+        paths = [p.numpy() for p in pr.paths]
+    threads = oracle.max_threads()
+    dtype = oracle.BF16 if small.path_dtype == "bf16" else oracle.F32
+
+    def step():
+        oracle.outer_sync(small.modules_per_level, small.level_numel, pr.table, theta, momentum,
+                          paths, dtype, float(np.float32(small.outer_lr)),
+                          float(np.float32(small.outer_momentum)), pr.weights, pr.reported, threads)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = small.path_params / dt
+    sample = ("each step: the oracle on %s parameters per level of all %d paths (%d path-params), "
+              "synthetic inputs drawn on the host" % ("/".join(str(x) for x in n), small.num_paths,
+                                                      small.path_params))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args):
+    import torch
+    from paper_2403_10616_b200 import binding as B
+    from paper_2403_10616_b200 import synth
+
+    world, rank, local = dist_setup(args)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the outer sync has no CPU path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    B.load()
+
+    cfg = workload_config(args)
+    need = cfg.path_params * (2 if cfg.path_dtype == "bf16" else 4) + 8 * cfg.module_params
+    free, _total = torch.cuda.mem_get_info(device)
+    if need * 1.02 > free:
+        raise SystemExit("workload needs %.1f GB of device memory, %.1f GB free" % (need / 1e9, free / 1e9))
+
+    problem = synth.make_problem(cfg, device)
+    torch.cuda.synchronize()
+    ptrs = [p.data_ptr() for p in problem.paths]
+    kernel = {"auto": B.DIPACO_KERNEL_AUTO, "vector": B.DIPACO_KERNEL_VECTOR,
+              "scalar": B.DIPACO_KERNEL_SCALAR}[args.kernel]
+    code = B.DIPACO_BF16 if cfg.path_dtype == "bf16" else B.DIPACO_F32
+
+    def make_ctx(chunk_paths):
+        ctx = B.dipaco_create(cfg.modules_per_level, cfg.level_numel, problem.table, problem.weights,
+                              np.float32(cfg.outer_lr), np.float32(cfg.outer_momentum), code,
+                              chunk_paths, local)
+        B.dipaco_set_kernel(ctx, kernel)
+        B.dipaco_set_tuning(ctx, args.ctas_per_sm, args.stages, args.units)
+        return ctx
+
+    # ---- resident one-pass mode: the headline value
+    ctx = make_ctx(0)
+
+    def step():
+        B.dipaco_outer_sync(ctx, problem.theta.data_ptr(), problem.momentum.data_ptr(), ptrs,
+                            problem.reported)
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    torch.cuda.synchronize()
+    launches_before = B.dipaco_launch_count(ctx)
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                           else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+    ms_region, ms_call = time_steps(step, args.steps, world)
+    clocks = sampler.stop()
+    launches = B.dipaco_launch_count(ctx) - launches_before
+    status = B.dipaco_device_status(ctx)
+    if status != B.DIPACO_OK:
+        raise SystemExit("device status after the timed region: %s" % B.strerror(status))
+    B.dipaco_destroy(ctx)
+
+    ms_max, units_total = aggregate(ms_region, float(cfg.path_params), world, device)
+    value = units_total / (ms_max * 1e-3)
+    alg_bytes = synth.algorithmic_bytes(cfg, problem.reported)
+    peak, peak_kind = measured_peak_hbm()
+    achieved = alg_bytes / (ms_call * 1e-3) / 1e9
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": cfg.name, "levels": list(cfg.modules_per_level),
+            "level_numel": list(cfg.level_numel), "paths": cfg.num_paths,
+            "path_dtype": cfg.path_dtype, "mode": "resident one-pass (all path copies in HBM)",
+            "l2": "inputs (%.1f GB) exceed L2, no flush between steps" % (need / 1e9),
+            "parallelism": "replicas only" if world > 1 else "1 GPU",
+            "kernel": args.kernel,
+        },
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "effective_gbs": achieved,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_kind": "of " + peak_kind,
+                     "kernel": "sync_bulk_kernel" if args.kernel == "auto" else "sync_direct_kernel",
+                     "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": ms_call,
+                     "frac_of_nominal_8tbs": achieved / 8000.0},
+    }
+
+    # ---- the same workload walked in chunks of paths (device resident)
+    if not args.no_chunked and cfg.chunk_paths > 0 and rank == 0:
+        ctx = make_ctx(cfg.chunk_paths)
+        for _ in range(max(args.warmup, 1)):
+            step_ctx = ctx
+            B.dipaco_outer_sync(step_ctx, problem.theta.data_ptr(), problem.momentum.data_ptr(), ptrs,
+                                problem.reported)
+        before = B.dipaco_launch_count(ctx)
+        ms_c, _ = time_steps(lambda: B.dipaco_outer_sync(ctx, problem.theta.data_ptr(),
+                                                         problem.momentum.data_ptr(), ptrs,
+                                                         problem.reported), args.steps, 1)
+        result["chunked"] = {"chunk_paths": cfg.chunk_paths, "ms_per_step": ms_c,
+                             "value": cfg.path_params / (ms_c * 1e-3), "unit": UNIT,
+                             "effective_gbs": alg_bytes / (ms_c * 1e-3) / 1e9,
+                             "gpu_launches": int(B.dipaco_launch_count(ctx) - before)}
+        B.dipaco_destroy(ctx)
+
+    # ---- CPU oracle on a slab of the same inputs (rank 0, N = 1)
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        result["cpu_baseline"] = cpu_baseline_from_device(problem, CPU_SAMPLE_NUMEL)
+
+    # ---- end to end through the host-buffer entry point
+    if not args.no_e2e:
+        result["e2e"] = run_e2e(args, cfg, problem, make_ctx, world, device)
+
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_e2e(args, cfg, problem, make_ctx, world, device):
+    """Same metric through dipaco_outer_sync_host: state in pinned host memory, every step copies
+    the inputs host->device and the results device->host inside the timed region."""
+    import torch
+    from paper_2403_10616_b200 import binding as B
+    chunk = cfg.chunk_paths if cfg.chunk_paths > 0 else min(32, cfg.num_paths)
+    es = 2 if cfg.path_dtype == "bf16" else 4
+    try:
+        theta_h = torch.empty_like(problem.theta, device="cpu").pin_memory()
+        mom_h = torch.empty_like(problem.momentum, device="cpu").pin_memory()
+        paths_h = torch.empty((cfg.num_paths, cfg.params_per_path), dtype=problem.paths[0].dtype,
+                              pin_memory=True)
+    except RuntimeError as exc:
+        return {"value": None, "unit": UNIT, "error": "could not pin host memory: %s" % exc}
+    theta_h.copy_(problem.theta)
+    mom_h.copy_(problem.momentum)
+    for i, p in enumerate(problem.paths):
+        paths_h[i].copy_(p)
+    torch.cuda.synchronize()
+    # the device copies are no longer needed: free them so the staging buffers fit
+    problem.paths.clear()
+    problem.storage = None
+    torch.cuda.empty_cache()
+    ctx = make_ctx(chunk)
+    hptrs = [paths_h[i].data_ptr() for i in range(cfg.num_paths)]
+
+    def step():
+        B.dipaco_outer_sync_host(ctx, theta_h.data_ptr(), mom_h.data_ptr(), hptrs, problem.reported)
+
+    step()   # warm-up: allocates the staging buffers
+    steps = max(1, args.e2e_steps)
+    barrier(world)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt_ms = (time.perf_counter() - t0) * 1e3 / steps
+    barrier(world)
+    ms_max, units = aggregate(dt_ms, float(cfg.path_params), world, device)
+    n_rep = cfg.num_paths if problem.reported is None else int(problem.reported.sum())
+    B.dipaco_destroy(ctx)
+    return {"value": units / (ms_max * 1e-3), "unit": UNIT, "ms_per_step": ms_max, "steps": steps,
+            "h2d_bytes_per_step": 8 * cfg.module_params + n_rep * cfg.params_per_path * es,
+            "d2h_bytes_per_step": 8 * cfg.module_params + cfg.num_paths * cfg.params_per_path * es,
+            "api": "dipaco_outer_sync_host, pinned host buffers, chunks of %d paths" % chunk}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,193 @@
+/*
+ * dipaco.h - C ABI of the module-wise outer synchronisation of DiPaCo on one CUDA device.
+ *
+ * The operation (DiPaCo, Algorithm 1, the outer-optimisation loop over levels and experts;
+ * Sections 2.5-2.7).  A model is a grid of L levels with K_l modules per level (Section 2.2);
+ * a path picks one module per level.  After the inner optimisation every path i holds its own
+ * copy x_i of each module it passes through.  For every module (l,e):
+ *
+ *     Delta = sum_{i in R(l,e)} c_i * (theta - x_i)            outer gradient, Algorithm 1
+ *     m'    = mu * m + Delta                                   Nesterov momentum (Section 2.5,
+ *     theta'= theta - lr * (Delta + mu * m')                    lr/mu: supplementary details)
+ *     x_i   = cast(theta')   for every path i through (l,e)    re-dispatch (Section 2.5)
+ *
+ * R(l,e) are the paths through (l,e) that reported this round (Section 2.6.2 trains subsets of
+ * paths; Section 3.1 describes preempted workers); c_i = w_i / sum_{j in R} w_j with w the raw
+ * per-path weights (shard sizes, Section 2.7 "Loss reweighing"; uniform when absent).  A module
+ * with no reporting path, or zero total weight, keeps theta and m bit for bit; its copies are
+ * still overwritten with cast(theta).  The reduction runs in ascending path id in fp32 with
+ * fused multiply-adds, so results are bitwise reproducible and identical between the resident
+ * and the chunked mode.
+ *
+ * Layouts.  theta and momentum: fp32, sum_l K_l*N_l elements ordered [level][module][element]
+ * (N_l = |B_l|, the size of every module of level l).  A path copy: sum_l N_l elements, the
+ * path's L modules concatenated in level order, fp32 or bf16 (round-to-nearest-even on write).
+ *
+ * Ownership.  The caller owns theta, momentum and all path buffers; they are updated in place.
+ * A context owns small device tables and, in chunked mode, an fp32 partial-sum scratch.
+ *
+ * Errors.  Every function returns a status (0 = ok, negative = error) and never throws, aborts
+ * or prints.  Arguments are validated before anything is launched: on a validation error the
+ * caller's buffers are untouched.  Calls are asynchronous on the given stream unless noted; all
+ * calls on one context must be ordered on one stream (or externally synchronised).
+ */
+#ifndef DIPACO_H
+#define DIPACO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dipaco_ctx dipaco_ctx;
+
+enum { DIPACO_F32 = 0, DIPACO_BF16 = 1 };
+
+enum {
+    DIPACO_OK = 0,
+    DIPACO_EINVAL = -1,   /* bad argument (null, out of range, non-finite, wrong state value)   */
+    DIPACO_ECUDA = -2,    /* a CUDA runtime call failed                                         */
+    DIPACO_ENOMEM = -3,   /* host or device allocation failed                                   */
+    DIPACO_ESTATE = -4,   /* call not allowed in the context's current state                    */
+    DIPACO_ETIMEOUT = -5, /* a bounded wait inside a kernel ran out (reported by device_status) */
+    DIPACO_ENODEV = -6    /* the context was created without a device (plan only)               */
+};
+
+/* kernel selection for dipaco_set_kernel */
+enum {
+    DIPACO_KERNEL_AUTO = 0,   /* bulk-copy (TMA) pipeline for 16-byte aligned full tiles, scalar rest */
+    DIPACO_KERNEL_VECTOR = 1, /* 128-bit register loads/stores for aligned full tiles, scalar rest    */
+    DIPACO_KERNEL_SCALAR = 2  /* one element per thread everywhere (any alignment)                    */
+};
+
+/*
+ * Build a context for one module grid (Algorithm 1, "Require" lines; Section 2.2 notation).
+ *   num_levels         L >= 1
+ *   modules_per_level  host [L], K_l >= 1
+ *   level_numel        host [L], N_l >= 0
+ *   num_paths          P >= 1; any set of paths, not only the full product (Section 2.6.2)
+ *   path_to_module     host [P*L] row-major, entry (i,l) in [0,K_l); a module no path uses is
+ *                      allowed and never touched (Section 2.6.1: any sharing pattern)
+ *   path_weights       host [P] raw weights >= 0, finite (Section 2.7), or NULL = uniform
+ *   outer_lr, outer_momentum   finite; the paper uses 0.7 and 0.9
+ *   path_dtype         DIPACO_F32 or DIPACO_BF16
+ *   chunk_paths        0 = all path copies are resident at once; c > 0 = copies are presented
+ *                      in chunks of c consecutive path ids (Section 3.3, online averaging)
+ *   device             CUDA device ordinal, or -1 for a plan-only context (no CUDA call is made;
+ *                      only the dipaco_plan_* queries work, everything else returns ENODEV)
+ * All host arrays are copied.  Synchronous.
+ */
+int dipaco_create(dipaco_ctx **out, int32_t num_levels, const int32_t *modules_per_level,
+                  const int64_t *level_numel, int32_t num_paths, const int32_t *path_to_module,
+                  const float *path_weights, float outer_lr, float outer_momentum,
+                  int32_t path_dtype, int32_t chunk_paths, int32_t device);
+
+/*
+ * One outer synchronisation of every module, in place (Algorithm 1, outer loop, plus re-dispatch).
+ *   theta, momentum  device, fp32, layout above; in/out
+ *   path_ptrs        HOST array [P] of DEVICE pointers, one per path copy; in/out
+ *   reported         HOST [P], nonzero = path i reported; NULL = all reported
+ *   cuda_stream      a cudaStream_t (0 = default stream)
+ * With chunk_paths = 0 this is one fused pass; otherwise the library walks the chunks
+ * (accumulate each chunk in ascending order, then write back) over the same device pointers.
+ */
+int dipaco_outer_sync(dipaco_ctx *ctx, float *theta, float *momentum, void *const *path_ptrs,
+                      const uint8_t *reported, void *cuda_stream);
+
+/*
+ * Incremental form of the same operation for callers that hold only one chunk of path copies
+ * on the device at a time (Section 3.3, "Online Parameter Gradient Averaging": each checkpoint
+ * is added to a partial sum as it arrives).  Requires chunk_paths > 0.  Chunk c covers path ids
+ * [c*chunk_paths, min(P, (c+1)*chunk_paths)).
+ *   begin      fixes theta, momentum, the mask and the stream for this round.
+ *   accumulate chunk_index must be 0,1,2,... in order; chunk_ptrs is a HOST array of the
+ *              chunk's DEVICE pointers.  Adds the chunk's reporting copies to the partial sums;
+ *              a module whose last reporting path lies in this chunk is updated right away and
+ *              written into this chunk's copies.
+ *   writeback  after every chunk has been accumulated, any order: fills every slot of the
+ *              chunk's copies with cast(theta') (the contents of chunk_ptrs are not read, so the
+ *              buffers may be fresh).
+ *   end        checks that every chunk was accumulated and returns the context to idle.
+ */
+int dipaco_sync_begin(dipaco_ctx *ctx, float *theta, float *momentum, const uint8_t *reported,
+                      void *cuda_stream);
+int dipaco_sync_accumulate(dipaco_ctx *ctx, int32_t chunk_index, void *const *chunk_ptrs);
+int dipaco_sync_writeback(dipaco_ctx *ctx, int32_t chunk_index, void *const *chunk_ptrs);
+int dipaco_sync_end(dipaco_ctx *ctx);
+
+/*
+ * The same synchronisation for state that lives in HOST memory (checkpoints that do not fit
+ * on the device): theta, momentum [module params] and the P path copies are host buffers
+ * (pinned memory gives full copy speed).  Path copies are streamed through the device in
+ * chunks of chunk_paths (> 0 required) with copies overlapping the kernels; theta' and m' are
+ * copied back and every path copy is overwritten with its modules' cast(theta').
+ * Synchronous: returns when all host buffers hold the result.
+ */
+int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
+                           void *const *path_ptrs_host, const uint8_t *reported,
+                           void *cuda_stream);
+
+/* Replace the raw per-path weights (host [P], or NULL = uniform).  Section 2.7. */
+int dipaco_set_weights(dipaco_ctx *ctx, const float *path_weights);
+
+/* Choose the kernel family (DIPACO_KERNEL_*); all families give bitwise identical results. */
+int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
+
+/*
+ * Tuning of the bulk-copy kernel: persistent CTAs per SM (1..8), pipeline depth in tiles (2..32)
+ * and 16-byte units of path data per compute thread and tile (1, 2 or 4; the tile is
+ * 256 threads * units * 16 bytes).  0 keeps a value.  A depth that does not fit the shared
+ * memory of the chosen layout is rejected with DIPACO_EINVAL and nothing changes.
+ */
+int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
+                      int32_t units_per_thread);
+
+/*
+ * Synchronise the context's last stream and report what the kernels recorded: DIPACO_OK, or
+ * DIPACO_ETIMEOUT if a bounded wait gave up (results of that call are then undefined), or
+ * DIPACO_ECUDA.  Clears the recorded status.
+ */
+int dipaco_device_status(dipaco_ctx *ctx);
+
+/* Number of kernels this context has launched so far. */
+int64_t dipaco_launch_count(const dipaco_ctx *ctx);
+
+/*
+ * Plan queries (host only; work on plan-only contexts too).  They expose step a0 of the path:
+ * the contributor set of a module under a mask and the normalised coefficients.
+ *   members / contributors  out, capacity num_paths each; ascending path ids
+ *   coeff                   out, capacity num_paths; c_i as the kernels use them (fp32)
+ *   will_update             out; 0 when no path reports or the total weight is zero
+ * Any out pointer may be NULL.
+ */
+int dipaco_plan_module(const dipaco_ctx *ctx, int32_t level, int32_t module,
+                       const uint8_t *reported, int32_t *num_members, int32_t *members,
+                       int32_t *num_contributors, int32_t *contributors, float *coeff,
+                       int32_t *will_update);
+/* Offsets (in elements) of module (level, module) in theta and of the level in a path copy. */
+int dipaco_plan_offsets(const dipaco_ctx *ctx, int32_t level, int32_t module,
+                        int64_t *theta_offset, int64_t *path_offset, int64_t *numel);
+/* Number of chunks (1 when chunk_paths = 0) and fp32 elements of partial-sum scratch. */
+int dipaco_plan_chunks(const dipaco_ctx *ctx, int32_t *num_chunks, int64_t *scratch_elems);
+
+/*
+ * The split of the resident-mode launch over num_ctas persistent CTAs in tiles of `tile`
+ * elements (all pointers assumed aligned): CTA b processes segments
+ * [cta_first[b], cta_first[b+1]); segment s covers elements [seg_begin[s], seg_end[s]) of
+ * module (seg_level[s], seg_module[s]).  Arrays have `capacity` entries (cta_first: num_ctas+1).
+ * Returns the number of segments (>= 0), or a negative status (EINVAL also when capacity is
+ * too small).
+ */
+int dipaco_plan_split(const dipaco_ctx *ctx, const uint8_t *reported, int32_t num_ctas, int64_t tile,
+                      int32_t capacity, int32_t *seg_level, int32_t *seg_module, int64_t *seg_begin,
+                      int64_t *seg_end, int32_t *cta_first);
+
+int dipaco_destroy(dipaco_ctx *ctx);
+
+const char *dipaco_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIPACO_H */

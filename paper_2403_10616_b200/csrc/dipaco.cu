@@ -1,0 +1,786 @@
+// C-ABI library of the module-wise outer synchronisation (see include/dipaco.h).
+// Host side: argument checks, planning (plan.hpp), table upload, kernel launches (kernels.cuh).
+#include "../../include/dipaco.h"
+
+#include <cstdio>
+#include <cstring>
+#include <functional>
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+#include "plan.hpp"
+
+using namespace dipaco;
+
+namespace {
+
+constexpr int STAGING_SLOTS = 4;
+constexpr size_t SMEM_LIMIT = 227 * 1024;  // opt-in dynamic shared memory per CTA on sm_100
+constexpr size_t SMEM_PER_SM = 228 * 1024;
+constexpr size_t SMEM_CTA_RESERVE = 1024;  // per-CTA reservation the driver adds
+constexpr int64_t RAGGED_TILE = 1024;      // split granularity of the scalar kernel
+
+enum SyncState { STATE_IDLE = 0, STATE_ACCUMULATING = 1 };
+
+struct Staging {
+    void *host = nullptr;
+    size_t capacity = 0;
+    cudaEvent_t done = nullptr;
+    bool in_flight = false;
+};
+
+// One kernel launch worth of tables inside a packed upload.
+struct PackedLaunch {
+    size_t passes_off = 0, contribs_off = 0, members_off = 0;
+    size_t bulk_segs_off = 0, bulk_first_off = 0, rag_segs_off = 0, rag_first_off = 0;
+    int bulk_ctas = 0, rag_ctas = 0;
+    int io_arrays = 2;
+    bool aligned_kernel_is_vector = false;
+};
+
+struct HostMode;  // state of dipaco_outer_sync_host (host_mode.inl)
+
+} // namespace
+
+struct dipaco_ctx {
+    Grid grid;
+    float lr = 0.f, mu = 0.f;
+    int dtype = DIPACO_F32;
+    int elem_size = 4;
+    int device = -1;
+    int sm_count = 0;
+    int kernel = DIPACO_KERNEL_AUTO;
+    int ctas_per_sm = 2, stages = 0, units = 0;  // 0 = automatic
+    int64_t launches = 0;
+
+    void *dev_tables = nullptr;
+    size_t dev_tables_capacity = 0;
+    Staging staging[STAGING_SLOTS];
+    int staging_next = 0;
+    float *partial = nullptr;
+    int *error_word = nullptr;
+    bool smem_attr_set[2][3] = {{false, false, false}, {false, false, false}};
+
+    // round state of the incremental API
+    int state = STATE_IDLE;
+    float *theta = nullptr, *momentum = nullptr;
+    cudaStream_t stream = nullptr;
+    cudaStream_t last_stream = nullptr;
+    std::vector<uint8_t> mask;       // copy of `reported` (empty = all reported)
+    std::vector<ModuleCoeffs> coeffs;
+    int next_chunk = 0;
+    std::vector<uint8_t> written_back;
+
+    HostMode *host_mode = nullptr;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+void compute_all_coeffs(dipaco_ctx *ctx, const uint8_t *reported)
+{
+    ctx->coeffs.resize(ctx->grid.modules.size());
+    for (size_t id = 0; id < ctx->grid.modules.size(); ++id)
+        module_coeffs(ctx->grid, ctx->grid.modules[id], reported, ctx->coeffs[id]);
+}
+
+int tile_units(const dipaco_ctx *ctx)
+{
+    if (ctx->units > 0) return ctx->units;
+    return ctx->dtype == DIPACO_BF16 ? 1 : 2;
+}
+
+int64_t tile_elems(const dipaco_ctx *ctx)
+{
+    const int ue = ctx->dtype == DIPACO_BF16 ? 8 : 4;
+    return (int64_t)BULK_COMPUTE_THREADS * ue * tile_units(ctx);
+}
+
+// Shared memory of one bulk-kernel CTA for a given depth.
+size_t bulk_smem_bytes(const dipaco_ctx *ctx, int stages, int io_arrays)
+{
+    const size_t tile = (size_t)tile_elems(ctx);
+    const size_t stage = tile * ctx->elem_size;
+    size_t bytes = (size_t)stages * stage + (size_t)2 * io_arrays * tile * 4;
+    if (ctx->elem_size != 4) bytes += 2 * stage;
+    return bytes + sizeof(BulkShared) + 128;
+}
+
+int pick_stages(const dipaco_ctx *ctx, int io_arrays)
+{
+    const size_t budget =
+        std::min(SMEM_LIMIT, SMEM_PER_SM / (size_t)ctx->ctas_per_sm - SMEM_CTA_RESERVE);
+    int best = 0;
+    for (int s = 2; s <= BULK_MAX_STAGES; ++s)
+        if (bulk_smem_bytes(ctx, s, io_arrays) <= budget) best = s;
+    if (ctx->stages > 0) return ctx->stages <= best ? ctx->stages : best;
+    return best;
+}
+
+struct PtrLookup {
+    void *const *ptrs;  // device pointers of path copies
+    int first_path;     // ptrs[0] belongs to this path id
+    int count;
+    void *get(int path) const
+    {
+        const int i = path - first_path;
+        return (i >= 0 && i < count) ? ptrs[i] : nullptr;
+    }
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Serialise the tables of one launch into `blob` (appending) and describe them in `out`.
+// extra_dst: optional raw destinations appended to a pass's member list (keyed by pass index).
+int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLookup &lookup,
+                const std::vector<std::vector<void *>> *extra_dst, const float *theta,
+                const float *momentum, std::vector<unsigned char> &blob, PackedLaunch &out)
+{
+    const Grid &g = ctx->grid;
+    const int es = ctx->elem_size;
+    std::vector<PassDev> passes(specs.size());
+    std::vector<ContribDev> contribs;
+    std::vector<void *> members;
+    std::vector<int64_t> bulk_begin(specs.size(), 0), bulk_end(specs.size(), 0);
+    std::vector<int64_t> rag_begin(specs.size(), 0), rag_end(specs.size(), 0);
+    const int64_t tile = tile_elems(ctx);
+    bool any_partial = false;
+
+    for (size_t i = 0; i < specs.size(); ++i) {
+        const PassSpec &sp = specs[i];
+        const ModuleGeom &m = g.modules[sp.module];
+        PassDev &pd = passes[i];
+        pd.theta_off = m.theta_off;
+        pd.partial_off = m.partial_off >= 0 ? m.partial_off : 0;
+        pd.flags = sp.flags;
+        pd.pad = 0;
+        if ((sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) && (m.partial_off < 0 || !ctx->partial))
+            return DIPACO_ESTATE;
+        if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
+        bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
+                       ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
+        pd.contrib_begin = (int)contribs.size();
+        for (size_t j = 0; j < sp.contributors.size(); ++j) {
+            char *base = static_cast<char *>(lookup.get(sp.contributors[j]));
+            if (!base) return DIPACO_EINVAL;
+            ContribDev c;
+            c.src = base + m.path_off * es;
+            c.coeff = sp.coeff[j];
+            c.pad = 0;
+            aligned = aligned && ((uintptr_t)c.src % 16 == 0);
+            contribs.push_back(c);
+        }
+        pd.contrib_count = (int)sp.contributors.size();
+        pd.member_begin = (int)members.size();
+        for (int path : sp.members) {
+            char *base = static_cast<char *>(lookup.get(path));
+            if (!base) return DIPACO_EINVAL;
+            void *dst = base + m.path_off * es;
+            aligned = aligned && ((uintptr_t)dst % 16 == 0);
+            members.push_back(dst);
+        }
+        if (extra_dst && i < extra_dst->size())
+            for (void *dst : (*extra_dst)[i]) {
+                aligned = aligned && ((uintptr_t)dst % 16 == 0);
+                members.push_back(dst);
+            }
+        pd.member_count = (int)members.size() - pd.member_begin;
+
+        int64_t full = 0;
+        if (aligned && ctx->kernel != DIPACO_KERNEL_SCALAR) full = m.numel / tile * tile;
+        bulk_begin[i] = 0; bulk_end[i] = full;
+        rag_begin[i] = full; rag_end[i] = m.numel;
+    }
+
+    std::vector<Segment> bulk_segs, rag_segs;
+    std::vector<int32_t> bulk_first, rag_first;
+    const bool vector_kernel = ctx->kernel == DIPACO_KERNEL_VECTOR;
+    int bulk_ctas = ctx->sm_count * (vector_kernel ? 8 : ctx->ctas_per_sm);
+    int64_t bulk_tiles = 0, rag_tiles = 0;
+    for (size_t i = 0; i < specs.size(); ++i) {
+        bulk_tiles += (bulk_end[i] - bulk_begin[i]) / tile;
+        rag_tiles += (rag_end[i] - rag_begin[i] + RAGGED_TILE - 1) / RAGGED_TILE;
+    }
+    if (bulk_tiles < bulk_ctas) bulk_ctas = (int)bulk_tiles;
+    int rag_ctas = (int)std::min<int64_t>(rag_tiles, (int64_t)ctx->sm_count * 8);
+    if (bulk_ctas > 0)
+        split_segments(specs, bulk_begin, bulk_end, es, tile, bulk_ctas, bulk_segs, bulk_first);
+    if (rag_ctas > 0)
+        split_segments(specs, rag_begin, rag_end, es, RAGGED_TILE, rag_ctas, rag_segs, rag_first);
+
+    auto append = [&](const void *src, size_t bytes) -> size_t {
+        const size_t off = align_up(blob.size(), 16);
+        blob.resize(off + bytes);
+        if (bytes) std::memcpy(blob.data() + off, src, bytes);
+        return off;
+    };
+    out.passes_off = append(passes.data(), passes.size() * sizeof(PassDev));
+    out.contribs_off = append(contribs.data(), contribs.size() * sizeof(ContribDev));
+    out.members_off = append(members.data(), members.size() * sizeof(void *));
+    static_assert(sizeof(Segment) == sizeof(SegmentDev), "segment layouts must match");
+    out.bulk_segs_off = append(bulk_segs.data(), bulk_segs.size() * sizeof(Segment));
+    out.bulk_first_off = append(bulk_first.data(), bulk_first.size() * sizeof(int32_t));
+    out.rag_segs_off = append(rag_segs.data(), rag_segs.size() * sizeof(Segment));
+    out.rag_first_off = append(rag_first.data(), rag_first.size() * sizeof(int32_t));
+    out.bulk_ctas = bulk_ctas;
+    out.rag_ctas = rag_ctas;
+    out.io_arrays = any_partial ? 3 : 2;
+    out.aligned_kernel_is_vector = vector_kernel;
+    return DIPACO_OK;
+}
+
+// Copy a packed blob to the device through a pinned staging slot (asynchronous on `stream`).
+int upload_blob(dipaco_ctx *ctx, const std::vector<unsigned char> &blob, cudaStream_t stream)
+{
+    const size_t bytes = std::max<size_t>(blob.size(), 16);
+    if (bytes > ctx->dev_tables_capacity) {
+        // grow: wait for earlier work that may still read the old tables
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return DIPACO_ECUDA;
+        if (ctx->last_stream && ctx->last_stream != stream &&
+            cudaStreamSynchronize(ctx->last_stream) != cudaSuccess)
+            return DIPACO_ECUDA;
+        if (ctx->dev_tables) cudaFree(ctx->dev_tables);
+        ctx->dev_tables = nullptr;
+        const size_t cap = align_up(bytes * 2, 4096);
+        if (cudaMalloc(&ctx->dev_tables, cap) != cudaSuccess) {
+            ctx->dev_tables_capacity = 0;
+            return DIPACO_ENOMEM;
+        }
+        ctx->dev_tables_capacity = cap;
+    }
+    Staging &st = ctx->staging[ctx->staging_next];
+    ctx->staging_next = (ctx->staging_next + 1) % STAGING_SLOTS;
+    if (st.in_flight) {
+        if (cudaEventSynchronize(st.done) != cudaSuccess) return DIPACO_ECUDA;
+        st.in_flight = false;
+    }
+    if (bytes > st.capacity) {
+        if (st.host) cudaFreeHost(st.host);
+        st.host = nullptr;
+        st.capacity = 0;
+        const size_t cap = align_up(bytes * 2, 4096);
+        if (cudaMallocHost(&st.host, cap) != cudaSuccess) return DIPACO_ENOMEM;
+        st.capacity = cap;
+    }
+    if (!st.done && cudaEventCreateWithFlags(&st.done, cudaEventDisableTiming) != cudaSuccess)
+        return DIPACO_ECUDA;
+    std::memcpy(st.host, blob.data(), blob.size());
+    if (cudaMemcpyAsync(ctx->dev_tables, st.host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return DIPACO_ECUDA;
+    if (cudaEventRecord(st.done, stream) != cudaSuccess) return DIPACO_ECUDA;
+    st.in_flight = true;
+    return DIPACO_OK;
+}
+
+template <typename PathT, int NU>
+int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages, int io_arrays,
+                  size_t smem, int attr_row, int attr_col, cudaStream_t stream)
+{
+    if (!ctx->smem_attr_set[attr_row][attr_col]) {
+        if (cudaFuncSetAttribute(sync_bulk_kernel<PathT, NU>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)SMEM_LIMIT) != cudaSuccess)
+            return DIPACO_ECUDA;
+        ctx->smem_attr_set[attr_row][attr_col] = true;
+    }
+    sync_bulk_kernel<PathT, NU><<<ctas, BULK_THREADS, smem, stream>>>(lp, stages, io_arrays);
+    return cudaGetLastError() == cudaSuccess ? DIPACO_OK : DIPACO_ECUDA;
+}
+
+int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays, cudaStream_t stream)
+{
+    const int stages = pick_stages(ctx, io_arrays);
+    if (stages < 2) return DIPACO_EINVAL;
+    const size_t smem = bulk_smem_bytes(ctx, stages, io_arrays);
+    const int nu = tile_units(ctx);
+    const int col = nu == 1 ? 0 : (nu == 2 ? 1 : 2);
+    if (ctx->dtype == DIPACO_BF16) {
+        if (nu == 1) return launch_bulk_t<__nv_bfloat16, 1>(ctx, lp, ctas, stages, io_arrays, smem, 1, col, stream);
+        if (nu == 2) return launch_bulk_t<__nv_bfloat16, 2>(ctx, lp, ctas, stages, io_arrays, smem, 1, col, stream);
+        return launch_bulk_t<__nv_bfloat16, 4>(ctx, lp, ctas, stages, io_arrays, smem, 1, col, stream);
+    }
+    if (nu == 1) return launch_bulk_t<float, 1>(ctx, lp, ctas, stages, io_arrays, smem, 0, col, stream);
+    if (nu == 2) return launch_bulk_t<float, 2>(ctx, lp, ctas, stages, io_arrays, smem, 0, col, stream);
+    return launch_bulk_t<float, 4>(ctx, lp, ctas, stages, io_arrays, smem, 0, col, stream);
+}
+
+int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *momentum,
+                  cudaStream_t stream)
+{
+    const char *base = static_cast<const char *>(ctx->dev_tables);
+    LaunchParams lp;
+    lp.theta = theta;
+    lp.momentum = momentum;
+    lp.partial = ctx->partial;
+    lp.passes = reinterpret_cast<const PassDev *>(base + pl.passes_off);
+    lp.contribs = reinterpret_cast<const ContribDev *>(base + pl.contribs_off);
+    lp.members = reinterpret_cast<void *const *>(base + pl.members_off);
+    lp.lr = ctx->lr;
+    lp.mu = ctx->mu;
+    lp.error_word = ctx->error_word;
+    if (pl.bulk_ctas > 0) {
+        lp.segs = reinterpret_cast<const SegmentDev *>(base + pl.bulk_segs_off);
+        lp.cta_first = reinterpret_cast<const int *>(base + pl.bulk_first_off);
+        int rc = DIPACO_OK;
+        if (pl.aligned_kernel_is_vector) {
+            if (ctx->dtype == DIPACO_BF16)
+                sync_direct_kernel<__nv_bfloat16, 8><<<pl.bulk_ctas, 256, 0, stream>>>(lp);
+            else
+                sync_direct_kernel<float, 8><<<pl.bulk_ctas, 256, 0, stream>>>(lp);
+            if (cudaGetLastError() != cudaSuccess) rc = DIPACO_ECUDA;
+        } else {
+            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, stream);
+        }
+        if (rc != DIPACO_OK) return rc;
+        ++ctx->launches;
+    }
+    if (pl.rag_ctas > 0) {
+        lp.segs = reinterpret_cast<const SegmentDev *>(base + pl.rag_segs_off);
+        lp.cta_first = reinterpret_cast<const int *>(base + pl.rag_first_off);
+        if (ctx->dtype == DIPACO_BF16)
+            sync_direct_kernel<__nv_bfloat16, 1><<<pl.rag_ctas, 256, 0, stream>>>(lp);
+        else
+            sync_direct_kernel<float, 1><<<pl.rag_ctas, 256, 0, stream>>>(lp);
+        if (cudaGetLastError() != cudaSuccess) return DIPACO_ECUDA;
+        ++ctx->launches;
+    }
+    return DIPACO_OK;
+}
+
+// Plan, upload and launch a list of launches that share one upload.
+struct LaunchRequest {
+    std::vector<PassSpec> specs;
+    PtrLookup lookup;
+    std::vector<std::vector<void *>> extra_dst;
+};
+
+int run_launches(dipaco_ctx *ctx, std::vector<LaunchRequest> &reqs, float *theta, float *momentum,
+                 cudaStream_t stream)
+{
+    std::vector<unsigned char> blob;
+    std::vector<PackedLaunch> packed(reqs.size());
+    for (size_t i = 0; i < reqs.size(); ++i) {
+        const int rc = pack_launch(ctx, reqs[i].specs, reqs[i].lookup,
+                                   reqs[i].extra_dst.empty() ? nullptr : &reqs[i].extra_dst, theta,
+                                   momentum, blob, packed[i]);
+        if (rc != DIPACO_OK) return rc;
+    }
+    int rc = upload_blob(ctx, blob, stream);
+    if (rc != DIPACO_OK) return rc;
+    for (size_t i = 0; i < reqs.size(); ++i) {
+        rc = launch_packed(ctx, packed[i], theta, momentum, stream);
+        if (rc != DIPACO_OK) return rc;
+    }
+    ctx->last_stream = stream;
+    return DIPACO_OK;
+}
+
+bool valid_ptr_array(void *const *ptrs, int n)
+{
+    if (!ptrs) return false;
+    for (int i = 0; i < n; ++i)
+        if (!ptrs[i]) return false;
+    return true;
+}
+
+int chunk_first(const Grid &g, int c) { return c * g.chunk_paths; }
+int chunk_count(const Grid &g, int c) { return std::min(g.chunk_paths, g.P - c * g.chunk_paths); }
+
+} // namespace
+
+#include "host_mode.inl"
+
+// ------------------------------------------------------------------------------------------ C ABI
+
+extern "C" {
+
+int dipaco_create(dipaco_ctx **out, int32_t num_levels, const int32_t *modules_per_level,
+                  const int64_t *level_numel, int32_t num_paths, const int32_t *path_to_module,
+                  const float *path_weights, float outer_lr, float outer_momentum,
+                  int32_t path_dtype, int32_t chunk_paths, int32_t device)
+{
+    if (!out) return DIPACO_EINVAL;
+    *out = nullptr;
+    if (path_dtype != DIPACO_F32 && path_dtype != DIPACO_BF16) return DIPACO_EINVAL;
+    if (!std::isfinite(outer_lr) || !std::isfinite(outer_momentum)) return DIPACO_EINVAL;
+    if (device < -1) return DIPACO_EINVAL;
+    dipaco_ctx *ctx = new (std::nothrow) dipaco_ctx();
+    if (!ctx) return DIPACO_ENOMEM;
+    try {
+        if (!build_grid(ctx->grid, num_levels, modules_per_level, level_numel, num_paths,
+                        path_to_module, path_weights, chunk_paths)) {
+            delete ctx;
+            return DIPACO_EINVAL;
+        }
+    } catch (const std::bad_alloc &) {
+        delete ctx;
+        return DIPACO_ENOMEM;
+    }
+    ctx->lr = outer_lr;
+    ctx->mu = outer_momentum;
+    ctx->dtype = path_dtype;
+    ctx->elem_size = path_dtype == DIPACO_BF16 ? 2 : 4;
+    ctx->device = device;
+    if (device >= 0) {
+        int count = 0;
+        if (cudaGetDeviceCount(&count) != cudaSuccess || device >= count) {
+            delete ctx;
+            return DIPACO_ECUDA;
+        }
+        DeviceGuard guard(device);
+        if (!guard.ok ||
+            cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+            delete ctx;
+            return DIPACO_ECUDA;
+        }
+        if (cudaMalloc(&ctx->error_word, sizeof(int)) != cudaSuccess ||
+            cudaMemset(ctx->error_word, 0, sizeof(int)) != cudaSuccess) {
+            dipaco_destroy(ctx);
+            return DIPACO_ENOMEM;
+        }
+        if (ctx->grid.scratch_elems > 0 &&
+            cudaMalloc(&ctx->partial, (size_t)ctx->grid.scratch_elems * sizeof(float)) != cudaSuccess) {
+            cudaGetLastError();
+            dipaco_destroy(ctx);
+            return DIPACO_ENOMEM;
+        }
+    }
+    *out = ctx;
+    return DIPACO_OK;
+}
+
+int dipaco_destroy(dipaco_ctx *ctx)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    int rc = DIPACO_OK;
+    if (ctx->device >= 0) {
+        DeviceGuard guard(ctx->device);
+        if (ctx->last_stream || ctx->stream) {
+            if (cudaStreamSynchronize(ctx->last_stream ? ctx->last_stream : ctx->stream) != cudaSuccess)
+                rc = DIPACO_ECUDA;
+        }
+        host_mode_release(ctx);
+        for (Staging &st : ctx->staging) {
+            if (st.done) cudaEventDestroy(st.done);
+            if (st.host) cudaFreeHost(st.host);
+        }
+        if (ctx->dev_tables) cudaFree(ctx->dev_tables);
+        if (ctx->partial) cudaFree(ctx->partial);
+        if (ctx->error_word) cudaFree(ctx->error_word);
+    }
+    delete ctx;
+    return rc;
+}
+
+int dipaco_set_weights(dipaco_ctx *ctx, const float *path_weights)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (path_weights) {
+        for (int i = 0; i < ctx->grid.P; ++i)
+            if (!(path_weights[i] >= 0.0f) || !std::isfinite(path_weights[i])) return DIPACO_EINVAL;
+        ctx->grid.weights.assign(path_weights, path_weights + ctx->grid.P);
+    } else {
+        ctx->grid.weights.clear();
+    }
+    return DIPACO_OK;
+}
+
+int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel)
+{
+    if (!ctx || kernel < DIPACO_KERNEL_AUTO || kernel > DIPACO_KERNEL_SCALAR) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ctx->kernel = kernel;
+    return DIPACO_OK;
+}
+
+int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int32_t units_per_thread)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (ctas_per_sm < 0 || ctas_per_sm > 8 || stages < 0 || stages == 1 || stages > BULK_MAX_STAGES)
+        return DIPACO_EINVAL;
+    if (units_per_thread != 0 && units_per_thread != 1 && units_per_thread != 2 && units_per_thread != 4)
+        return DIPACO_EINVAL;
+    const int old_ctas = ctx->ctas_per_sm, old_units = ctx->units, old_stages = ctx->stages;
+    if (ctas_per_sm) ctx->ctas_per_sm = ctas_per_sm;
+    if (units_per_thread) ctx->units = units_per_thread;
+    ctx->stages = 0;
+    const bool fits = pick_stages(ctx, 3) >= 2 && (!stages || stages <= pick_stages(ctx, 2));
+    if (!fits) {
+        ctx->ctas_per_sm = old_ctas;
+        ctx->units = old_units;
+        ctx->stages = old_stages;
+        return DIPACO_EINVAL;
+    }
+    ctx->stages = stages ? stages : old_stages;
+    return DIPACO_OK;
+}
+
+int dipaco_sync_begin(dipaco_ctx *ctx, float *theta, float *momentum, const uint8_t *reported,
+                      void *cuda_stream)
+{
+    if (!ctx || !theta || !momentum) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (ctx->grid.chunk_paths <= 0) return DIPACO_ESTATE;
+    try {
+        if (reported) ctx->mask.assign(reported, reported + ctx->grid.P);
+        else ctx->mask.clear();
+        compute_all_coeffs(ctx, reported);
+        ctx->written_back.assign((size_t)ctx->grid.num_chunks, 0);
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+    ctx->theta = theta;
+    ctx->momentum = momentum;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->next_chunk = 0;
+    ctx->state = STATE_ACCUMULATING;
+    return DIPACO_OK;
+}
+
+int dipaco_sync_accumulate(dipaco_ctx *ctx, int32_t chunk_index, void *const *chunk_ptrs)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_ACCUMULATING) return DIPACO_ESTATE;
+    if (chunk_index != ctx->next_chunk || chunk_index >= ctx->grid.num_chunks) return DIPACO_ESTATE;
+    const int n = chunk_count(ctx->grid, chunk_index);
+    if (!valid_ptr_array(chunk_ptrs, n)) return DIPACO_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DIPACO_ECUDA;
+    try {
+        std::vector<LaunchRequest> reqs(1);
+        plan_accumulate(ctx->grid, ctx->coeffs, chunk_index, reqs[0].specs);
+        reqs[0].lookup = PtrLookup{chunk_ptrs, chunk_first(ctx->grid, chunk_index), n};
+        if (!reqs[0].specs.empty()) {
+            const int rc = run_launches(ctx, reqs, ctx->theta, ctx->momentum, ctx->stream);
+            if (rc != DIPACO_OK) return rc;
+        }
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+    ++ctx->next_chunk;
+    return DIPACO_OK;
+}
+
+int dipaco_sync_writeback(dipaco_ctx *ctx, int32_t chunk_index, void *const *chunk_ptrs)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_ACCUMULATING || ctx->next_chunk != ctx->grid.num_chunks) return DIPACO_ESTATE;
+    if (chunk_index < 0 || chunk_index >= ctx->grid.num_chunks) return DIPACO_EINVAL;
+    const int n = chunk_count(ctx->grid, chunk_index);
+    if (!valid_ptr_array(chunk_ptrs, n)) return DIPACO_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DIPACO_ECUDA;
+    try {
+        std::vector<LaunchRequest> reqs(1);
+        plan_writeback(ctx->grid, ctx->coeffs, chunk_index, false, reqs[0].specs);
+        reqs[0].lookup = PtrLookup{chunk_ptrs, chunk_first(ctx->grid, chunk_index), n};
+        if (!reqs[0].specs.empty()) {
+            const int rc = run_launches(ctx, reqs, ctx->theta, ctx->momentum, ctx->stream);
+            if (rc != DIPACO_OK) return rc;
+        }
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+    ctx->written_back[(size_t)chunk_index] = 1;
+    return DIPACO_OK;
+}
+
+int dipaco_sync_end(dipaco_ctx *ctx)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_ACCUMULATING) return DIPACO_ESTATE;
+    const bool complete = ctx->next_chunk == ctx->grid.num_chunks;
+    ctx->state = STATE_IDLE;
+    return complete ? DIPACO_OK : DIPACO_ESTATE;
+}
+
+int dipaco_outer_sync(dipaco_ctx *ctx, float *theta, float *momentum, void *const *path_ptrs,
+                      const uint8_t *reported, void *cuda_stream)
+{
+    if (!ctx || !theta || !momentum) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (!valid_ptr_array(path_ptrs, ctx->grid.P)) return DIPACO_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DIPACO_ECUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const Grid &g = ctx->grid;
+    try {
+        compute_all_coeffs(ctx, reported);
+        std::vector<LaunchRequest> reqs;
+        if (g.num_chunks <= 1) {
+            reqs.resize(1);
+            plan_resident(g, ctx->coeffs, reqs[0].specs);
+            reqs[0].lookup = PtrLookup{path_ptrs, 0, g.P};
+        } else {
+            // accumulate every chunk in ascending order, then fill the slots that were not final yet
+            for (int c = 0; c < g.num_chunks; ++c) {
+                LaunchRequest r;
+                plan_accumulate(g, ctx->coeffs, c, r.specs);
+                r.lookup = PtrLookup{path_ptrs + chunk_first(g, c), chunk_first(g, c), chunk_count(g, c)};
+                if (!r.specs.empty()) reqs.push_back(std::move(r));
+            }
+            for (int c = 0; c < g.num_chunks; ++c) {
+                LaunchRequest r;
+                plan_writeback(g, ctx->coeffs, c, true, r.specs);
+                r.lookup = PtrLookup{path_ptrs + chunk_first(g, c), chunk_first(g, c), chunk_count(g, c)};
+                if (!r.specs.empty()) reqs.push_back(std::move(r));
+            }
+        }
+        bool any = false;
+        for (auto &r : reqs) any = any || !r.specs.empty();
+        if (!any) return DIPACO_OK;
+        return run_launches(ctx, reqs, theta, momentum, stream);
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+}
+
+int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
+                           void *const *path_ptrs_host, const uint8_t *reported, void *cuda_stream)
+{
+    if (!ctx || !theta_host || !momentum_host) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (ctx->grid.chunk_paths <= 0) return DIPACO_ESTATE;
+    if (!valid_ptr_array(path_ptrs_host, ctx->grid.P)) return DIPACO_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DIPACO_ECUDA;
+    try {
+        return host_mode_sync(ctx, theta_host, momentum_host, path_ptrs_host, reported,
+                              static_cast<cudaStream_t>(cuda_stream));
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+}
+
+int dipaco_device_status(dipaco_ctx *ctx)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DIPACO_ECUDA;
+    cudaStream_t s = ctx->last_stream ? ctx->last_stream : ctx->stream;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return DIPACO_ECUDA;
+    int word = 0;
+    if (cudaMemcpy(&word, ctx->error_word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return DIPACO_ECUDA;
+    if (word != 0) {
+        cudaMemset(ctx->error_word, 0, sizeof(int));
+        return DIPACO_ETIMEOUT;
+    }
+    return DIPACO_OK;
+}
+
+int64_t dipaco_launch_count(const dipaco_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int dipaco_plan_module(const dipaco_ctx *ctx, int32_t level, int32_t module, const uint8_t *reported,
+                       int32_t *num_members, int32_t *members, int32_t *num_contributors,
+                       int32_t *contributors, float *coeff, int32_t *will_update)
+{
+    if (!ctx || level < 0 || level >= ctx->grid.L || module < 0 || module >= ctx->grid.K[level])
+        return DIPACO_EINVAL;
+    try {
+        const ModuleGeom &m = ctx->grid.modules[ctx->grid.module_id(level, module)];
+        ModuleCoeffs mc;
+        module_coeffs(ctx->grid, m, reported, mc);
+        if (num_members) *num_members = (int32_t)m.members.size();
+        if (members) std::copy(m.members.begin(), m.members.end(), members);
+        if (num_contributors) *num_contributors = (int32_t)mc.contributors.size();
+        if (contributors) std::copy(mc.contributors.begin(), mc.contributors.end(), contributors);
+        if (coeff) std::copy(mc.coeff.begin(), mc.coeff.end(), coeff);
+        if (will_update) *will_update = mc.update ? 1 : 0;
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+    return DIPACO_OK;
+}
+
+int dipaco_plan_offsets(const dipaco_ctx *ctx, int32_t level, int32_t module, int64_t *theta_offset,
+                        int64_t *path_offset, int64_t *numel)
+{
+    if (!ctx || level < 0 || level >= ctx->grid.L || module < 0 || module >= ctx->grid.K[level])
+        return DIPACO_EINVAL;
+    const ModuleGeom &m = ctx->grid.modules[ctx->grid.module_id(level, module)];
+    if (theta_offset) *theta_offset = m.theta_off;
+    if (path_offset) *path_offset = m.path_off;
+    if (numel) *numel = m.numel;
+    return DIPACO_OK;
+}
+
+int dipaco_plan_chunks(const dipaco_ctx *ctx, int32_t *num_chunks, int64_t *scratch_elems)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (num_chunks) *num_chunks = ctx->grid.num_chunks;
+    if (scratch_elems) *scratch_elems = ctx->grid.scratch_elems;
+    return DIPACO_OK;
+}
+
+int dipaco_plan_split(const dipaco_ctx *ctx, const uint8_t *reported, int32_t num_ctas, int64_t tile,
+                      int32_t capacity, int32_t *seg_level, int32_t *seg_module, int64_t *seg_begin,
+                      int64_t *seg_end, int32_t *cta_first)
+{
+    if (!ctx || num_ctas < 1 || tile < 1 || capacity < 0) return DIPACO_EINVAL;
+    try {
+        std::vector<ModuleCoeffs> mc(ctx->grid.modules.size());
+        for (size_t id = 0; id < mc.size(); ++id)
+            module_coeffs(ctx->grid, ctx->grid.modules[id], reported, mc[id]);
+        std::vector<PassSpec> specs;
+        plan_resident(ctx->grid, mc, specs);
+        std::vector<int64_t> begin(specs.size(), 0), end(specs.size(), 0);
+        for (size_t i = 0; i < specs.size(); ++i)
+            end[i] = ctx->grid.modules[specs[i].module].numel / tile * tile;
+        std::vector<Segment> segs;
+        std::vector<int32_t> first;
+        split_segments(specs, begin, end, ctx->elem_size, tile, num_ctas, segs, first);
+        if ((int64_t)segs.size() > capacity) return DIPACO_EINVAL;
+        for (size_t s = 0; s < segs.size(); ++s) {
+            const ModuleGeom &m = ctx->grid.modules[specs[segs[s].pass].module];
+            if (seg_level) seg_level[s] = m.level;
+            if (seg_module) seg_module[s] = m.index;
+            if (seg_begin) seg_begin[s] = segs[s].begin;
+            if (seg_end) seg_end[s] = segs[s].end;
+        }
+        if (cta_first)
+            for (int b = 0; b <= num_ctas; ++b) cta_first[b] = first[(size_t)b];
+        return (int)segs.size();
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+}
+
+const char *dipaco_strerror(int status)
+{
+    switch (status) {
+    case DIPACO_OK: return "ok";
+    case DIPACO_EINVAL: return "invalid argument";
+    case DIPACO_ECUDA: return "CUDA runtime call failed";
+    case DIPACO_ENOMEM: return "out of memory";
+    case DIPACO_ESTATE: return "call not allowed in this state";
+    case DIPACO_ETIMEOUT: return "a bounded wait inside a kernel ran out";
+    case DIPACO_ENODEV: return "context has no device (plan only)";
+    default: return "unknown status";
+    }
+}
+
+} // extern "C"

@@ -1,0 +1,665 @@
+// Device code of the outer synchronisation (DiPaCo, Algorithm 1, outer loop + re-dispatch).
+//
+// Three kernel families share one arithmetic definition (sync_math below), so they give
+// bitwise identical results:
+//   sync_direct_kernel<PathT,1>   one element per thread, any alignment (ragged tails, odd offsets)
+//   sync_direct_kernel<PathT,8>   128-bit register loads/stores on 16-byte aligned full tiles
+//   sync_bulk_kernel<PathT,NU>    persistent, warp-specialised: one warp streams tiles into a
+//                                 shared-memory ring with bulk async copies (TMA, 1-D), eight
+//                                 warps reduce + apply Nesterov, one warp scatters the result
+//                                 tile to every path with bulk stores from shared memory.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dipaco {
+
+enum : int { KPASS_UPDATE = 1, KPASS_PARTIAL_IN = 2, KPASS_PARTIAL_OUT = 4 };
+
+struct PassDev {
+    long long theta_off;    // elements into theta / momentum
+    long long partial_off;  // elements into the partial-sum scratch (valid with PARTIAL flags)
+    int contrib_begin, contrib_count;
+    int member_begin, member_count;
+    int flags, pad;
+};
+
+struct ContribDev {
+    const void *src;  // start of the module's slot inside the contributor's path copy
+    float coeff;      // c_i = w_i / W
+    int pad;
+};
+
+struct SegmentDev {
+    int pass, pad;
+    long long begin, end;  // element range inside the module
+};
+
+struct LaunchParams {
+    float *theta;
+    float *momentum;
+    float *partial;
+    const PassDev *passes;
+    const ContribDev *contribs;
+    void *const *members;  // start of the module's slot inside each member path copy
+    const SegmentDev *segs;
+    const int *cta_first;  // [gridDim.x + 1]
+    float lr, mu;
+    int *error_word;
+};
+
+// ------------------------------------------------------------------------------------------
+// The arithmetic, written once.  Explicit intrinsics: no contraction or reassociation choices
+// are left to the compiler, so every kernel family rounds identically.
+
+__device__ __forceinline__ float sync_accumulate(float acc, float c, float theta, float x)
+{
+    // acc + c * (theta - x): one term of the outer gradient (Algorithm 1, outer-gradient line)
+    return __fmaf_rn(c, __fsub_rn(theta, x), acc);
+}
+
+__device__ __forceinline__ void sync_nesterov(float theta, float m, float delta, float lr, float mu,
+                                              float &theta_new, float &m_new)
+{
+    // m' = mu*m + Delta ; theta' = theta - lr*(Delta + mu*m')
+    m_new = __fmaf_rn(mu, m, delta);
+    const float g = __fmaf_rn(mu, m_new, delta);
+    theta_new = __fmaf_rn(-lr, g, theta);
+}
+
+template <typename T> struct PathIO;
+
+template <> struct PathIO<float> {
+    static __device__ __forceinline__ float load(const float *p) { return __ldcs(p); }
+    static __device__ __forceinline__ void store(float *p, float v) { __stcs(p, v); }
+};
+
+template <> struct PathIO<__nv_bfloat16> {
+    static __device__ __forceinline__ float load(const __nv_bfloat16 *p)
+    {
+        const unsigned short bits = __ldcs(reinterpret_cast<const unsigned short *>(p));
+        return __uint_as_float(((unsigned)bits) << 16);
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, float v)
+    {
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        __stcs(reinterpret_cast<unsigned short *>(p), __bfloat16_as_ushort(h));
+    }
+};
+
+// 16 bytes of path data <-> floats.  UE = elements per 16-byte unit.
+template <typename T> struct Unit;
+
+template <> struct Unit<float> {
+    static constexpr int UE = 4;
+    static __device__ __forceinline__ void widen(const uint4 &v, float *f)
+    {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ uint4 narrow(const float *f)
+    {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                          __float_as_uint(f[3]));
+    }
+};
+
+template <> struct Unit<__nv_bfloat16> {
+    static constexpr int UE = 8;
+    static __device__ __forceinline__ void widen(const uint4 &v, float *f)
+    {
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ unsigned pack(float lo, float hi)
+    {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);  // .x = lo (low half), .y = hi
+        return *reinterpret_cast<const unsigned *>(&h);
+    }
+    static __device__ __forceinline__ uint4 narrow(const float *f)
+    {
+        return make_uint4(pack(f[0], f[1]), pack(f[2], f[3]), pack(f[4], f[5]), pack(f[6], f[7]));
+    }
+};
+
+// ------------------------------------------------------------------------------------------
+// Direct kernels: every thread owns VEC consecutive elements and walks the contributors itself.
+
+template <typename PathT, int VEC>
+__global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
+{
+    const int seg_begin = p.cta_first[blockIdx.x];
+    const int seg_end = p.cta_first[blockIdx.x + 1];
+    for (int s = seg_begin; s < seg_end; ++s) {
+        const SegmentDev seg = p.segs[s];
+        const PassDev pass = p.passes[seg.pass];
+        const ContribDev *contribs = p.contribs + pass.contrib_begin;
+        void *const *members = p.members + pass.member_begin;
+        float *theta = p.theta + pass.theta_off;
+        float *momentum = p.momentum + pass.theta_off;
+        float *partial = p.partial + pass.partial_off;
+
+        for (long long k = seg.begin + (long long)threadIdx.x * VEC; k < seg.end;
+             k += (long long)blockDim.x * VEC) {
+            float th[VEC], acc[VEC];
+            if constexpr (VEC == 1) {
+                th[0] = theta[k];
+                acc[0] = (pass.flags & KPASS_PARTIAL_IN) ? partial[k] : 0.0f;
+                for (int j = 0; j < pass.contrib_count; ++j) {
+                    const ContribDev c = contribs[j];
+                    const float x = PathIO<PathT>::load(static_cast<const PathT *>(c.src) + k);
+                    acc[0] = sync_accumulate(acc[0], c.coeff, th[0], x);
+                }
+            } else {
+                constexpr int UE = Unit<PathT>::UE;
+                constexpr int UNITS = VEC / UE;  // 16-byte loads per contributor
+                constexpr int BATCH = 8 / UNITS; // contributors whose loads are issued together
+#pragma unroll
+                for (int v = 0; v < VEC; v += 4) {
+                    const float4 t = *reinterpret_cast<const float4 *>(theta + k + v);
+                    th[v] = t.x; th[v + 1] = t.y; th[v + 2] = t.z; th[v + 3] = t.w;
+                }
+                if (pass.flags & KPASS_PARTIAL_IN) {
+#pragma unroll
+                    for (int v = 0; v < VEC; v += 4) {
+                        const float4 t = *reinterpret_cast<const float4 *>(partial + k + v);
+                        acc[v] = t.x; acc[v + 1] = t.y; acc[v + 2] = t.z; acc[v + 3] = t.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VEC; ++v) acc[v] = 0.0f;
+                }
+                for (int j0 = 0; j0 < pass.contrib_count; j0 += BATCH) {
+                    uint4 raw[BATCH][UNITS];
+                    float coeff[BATCH];
+#pragma unroll
+                    for (int b = 0; b < BATCH; ++b) {
+                        if (j0 + b < pass.contrib_count) {
+                            const ContribDev c = contribs[j0 + b];
+                            coeff[b] = c.coeff;
+                            const uint4 *src = reinterpret_cast<const uint4 *>(
+                                static_cast<const PathT *>(c.src) + k);
+#pragma unroll
+                            for (int u = 0; u < UNITS; ++u) raw[b][u] = __ldcs(src + u);
+                        }
+                    }
+#pragma unroll
+                    for (int b = 0; b < BATCH; ++b) {
+                        if (j0 + b < pass.contrib_count) {
+#pragma unroll
+                            for (int u = 0; u < UNITS; ++u) {
+                                float x[UE];
+                                Unit<PathT>::widen(raw[b][u], x);
+#pragma unroll
+                                for (int i = 0; i < UE; ++i)
+                                    acc[u * UE + i] =
+                                        sync_accumulate(acc[u * UE + i], coeff[b], th[u * UE + i], x[i]);
+                            }
+                        }
+                    }
+                }
+            }
+
+            if (pass.flags & KPASS_PARTIAL_OUT) {
+                if constexpr (VEC == 1) {
+                    partial[k] = acc[0];
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VEC; v += 4)
+                        *reinterpret_cast<float4 *>(partial + k + v) =
+                            make_float4(acc[v], acc[v + 1], acc[v + 2], acc[v + 3]);
+                }
+            }
+            if (pass.flags & KPASS_UPDATE) {
+                float mo[VEC];
+                if constexpr (VEC == 1) {
+                    mo[0] = momentum[k];
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VEC; v += 4) {
+                        const float4 t = *reinterpret_cast<const float4 *>(momentum + k + v);
+                        mo[v] = t.x; mo[v + 1] = t.y; mo[v + 2] = t.z; mo[v + 3] = t.w;
+                    }
+                }
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) {
+                    float t1, m1;
+                    sync_nesterov(th[v], mo[v], acc[v], p.lr, p.mu, t1, m1);
+                    th[v] = t1;
+                    mo[v] = m1;
+                }
+                if constexpr (VEC == 1) {
+                    theta[k] = th[0];
+                    momentum[k] = mo[0];
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VEC; v += 4) {
+                        *reinterpret_cast<float4 *>(theta + k + v) =
+                            make_float4(th[v], th[v + 1], th[v + 2], th[v + 3]);
+                        *reinterpret_cast<float4 *>(momentum + k + v) =
+                            make_float4(mo[v], mo[v + 1], mo[v + 2], mo[v + 3]);
+                    }
+                }
+            }
+            if (pass.member_count > 0) {
+                if constexpr (VEC == 1) {
+                    for (int j = 0; j < pass.member_count; ++j)
+                        PathIO<PathT>::store(static_cast<PathT *>(members[j]) + k, th[0]);
+                } else {
+                    constexpr int UE = Unit<PathT>::UE;
+                    constexpr int UNITS = VEC / UE;
+                    uint4 out[UNITS];
+#pragma unroll
+                    for (int u = 0; u < UNITS; ++u) out[u] = Unit<PathT>::narrow(th + u * UE);
+                    for (int j = 0; j < pass.member_count; ++j) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(static_cast<PathT *>(members[j]) + k);
+#pragma unroll
+                        for (int u = 0; u < UNITS; ++u) __stcs(dst + u, out[u]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Bulk-copy (TMA) pipeline.
+
+namespace ptx {
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// global -> shared bulk copy, completion signalled on an mbarrier (bytes: multiple of 16)
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, unsigned bytes,
+                                          uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(smem_addr(dst_smem)),
+        "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+// shared -> global bulk copy, tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void bulk_store(void *dst_gmem, const void *src_smem, unsigned bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst_gmem),
+                 "r"(smem_addr(src_smem)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+} // namespace ptx
+
+constexpr int BULK_COMPUTE_WARPS = 8;
+constexpr int BULK_COMPUTE_THREADS = BULK_COMPUTE_WARPS * 32;
+constexpr int BULK_THREADS = BULK_COMPUTE_THREADS + 64;  // + load warp + store warp
+constexpr int BULK_MAX_STAGES = 32;
+constexpr unsigned long long BULK_WAIT_LIMIT_NS = 4000000000ull;  // every wait gives up after 4 s
+
+// Bounded wait: returns false (and records the failure) if the phase does not complete in time.
+__device__ __forceinline__ bool bounded_wait(uint64_t *bar, unsigned parity, int *error_word, int code)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = ptx::global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (ptx::global_timer_ns() - t0 > BULK_WAIT_LIMIT_NS) {
+            atomicCAS(error_word, 0, code);
+            return false;
+        }
+    }
+}
+
+struct BulkShared {
+    uint64_t full[BULK_MAX_STAGES];   // ring slot filled by a bulk load
+    uint64_t empty[BULK_MAX_STAGES];  // ring slot released by the compute warps
+    uint64_t io_full[2];              // theta / momentum / partial tiles loaded
+    uint64_t io_empty[2];             // result tiles drained by the store warp
+    uint64_t out_ready[2];            // compute warps finished writing the result tiles
+    float slot_coeff[BULK_MAX_STAGES];
+    const void *batch_src[32];
+    float batch_coeff[32];
+};
+
+// Position in the shared-memory ring: slot index and the phase parity of its barriers.
+struct RingPos {
+    int slot = 0;
+    unsigned phase = 0;
+    unsigned used = 0;  // slots used so far
+    __device__ __forceinline__ void advance(int stages)
+    {
+        ++used;
+        if (++slot == stages) { slot = 0; phase ^= 1u; }
+    }
+    __device__ __forceinline__ void retreat(int stages)
+    {
+        --used;
+        if (slot == 0) { slot = stages - 1; phase ^= 1u; } else { --slot; }
+    }
+};
+
+// Tile walk shared by the three roles: every role visits the same (pass, first element) sequence.
+struct TileWalk {
+    const SegmentDev *segs;
+    int seg, seg_end;
+    long long pos, end;
+    int pass;
+    long long tile;
+    __device__ TileWalk(const LaunchParams &p, long long tile_elems)
+        : segs(p.segs), seg(p.cta_first[blockIdx.x]), seg_end(p.cta_first[blockIdx.x + 1]), pos(0),
+          end(0), pass(-1), tile(tile_elems)
+    {
+        seg -= 1;
+    }
+    __device__ bool next(long long &k0)
+    {
+        if (pass >= 0) pos += tile;
+        while (pass < 0 || pos >= end) {
+            if (++seg >= seg_end) return false;
+            const SegmentDev s = segs[seg];
+            pass = s.pass; pos = s.begin; end = s.end;
+        }
+        k0 = pos;
+        return true;
+    }
+};
+
+// NU = 16-byte units of path data per compute thread and tile; tile = 256 * NU * UE elements.
+template <typename PathT, int NU>
+__global__ void __launch_bounds__(BULK_THREADS, 1)
+sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
+{
+    constexpr int UE = Unit<PathT>::UE;
+    constexpr int EPT = UE * NU;                         // elements per compute thread
+    constexpr int TILE = BULK_COMPUTE_THREADS * EPT;     // elements per tile
+    constexpr unsigned STAGE_BYTES = TILE * sizeof(PathT);
+    constexpr unsigned F32_TILE_BYTES = TILE * 4u;
+    constexpr bool NEED_CAST_TILE = sizeof(PathT) != 4;
+
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // layout: ring | io[2][io_arrays] fp32 tiles | cast tile[2] (bf16 only) | BulkShared
+    unsigned char *ring = smem_raw;
+    unsigned char *io = ring + (size_t)stages * STAGE_BYTES;
+    unsigned char *cast_tiles = io + (size_t)2 * io_arrays * F32_TILE_BYTES;
+    BulkShared *sh = reinterpret_cast<BulkShared *>(cast_tiles + (NEED_CAST_TILE ? 2u * STAGE_BYTES : 0u));
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(&sh->full[s], 1);
+            ptx::mbar_init(&sh->empty[s], BULK_COMPUTE_WARPS);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&sh->io_full[b], 1);
+            ptx::mbar_init(&sh->io_empty[b], 1);
+            ptx::mbar_init(&sh->out_ready[b], BULK_COMPUTE_WARPS);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    auto io_tile = [&](int b, int which) -> float * {
+        return reinterpret_cast<float *>(io + ((size_t)b * io_arrays + which) * F32_TILE_BYTES);
+    };
+    // io tile roles: 0 = theta (becomes theta'), 1 = momentum (becomes m'), 2 = partial sum
+    auto cast_tile = [&](int b) -> unsigned char * {
+        return NEED_CAST_TILE ? cast_tiles + (size_t)b * STAGE_BYTES
+                              : reinterpret_cast<unsigned char *>(io_tile(b, 0));
+    };
+
+    TileWalk walk(p, TILE);
+    long long k0;
+    unsigned t = 0;  // tiles seen by this role
+    RingPos q;       // ring position of this role
+
+    if (warp == BULK_COMPUTE_WARPS) {
+        // ------------------------------------------------------------------ load warp
+        bool ok = true;
+        while (ok && walk.next(k0)) {
+            const PassDev pass = p.passes[walk.pass];
+            const int b = t & 1;
+            if (lane == 0) {
+                ok = bounded_wait(&sh->io_empty[b], ((t >> 1) & 1) ^ 1, p.error_word, 1);
+                if (ok) {
+                    unsigned bytes = F32_TILE_BYTES;
+                    if (pass.flags & KPASS_UPDATE) bytes += F32_TILE_BYTES;
+                    if (pass.flags & KPASS_PARTIAL_IN) bytes += F32_TILE_BYTES;
+                    ptx::mbar_arrive_expect_tx(&sh->io_full[b], bytes);
+                    ptx::bulk_load(io_tile(b, 0), p.theta + pass.theta_off + k0, F32_TILE_BYTES,
+                                   &sh->io_full[b]);
+                    if (pass.flags & KPASS_UPDATE)
+                        ptx::bulk_load(io_tile(b, 1), p.momentum + pass.theta_off + k0,
+                                       F32_TILE_BYTES, &sh->io_full[b]);
+                    if (pass.flags & KPASS_PARTIAL_IN)
+                        ptx::bulk_load(io_tile(b, 2), p.partial + pass.partial_off + k0,
+                                       F32_TILE_BYTES, &sh->io_full[b]);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            for (int j0 = 0; ok && j0 < pass.contrib_count; j0 += 32) {
+                const int cnt = min(32, pass.contrib_count - j0);
+                if (lane < cnt) {
+                    const ContribDev c = p.contribs[pass.contrib_begin + j0 + lane];
+                    sh->batch_src[lane] = c.src;
+                    sh->batch_coeff[lane] = c.coeff;
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    for (int u = 0; u < cnt; ++u) {
+                        const int s = q.slot;
+                        ok = bounded_wait(&sh->empty[s], q.phase ^ 1u, p.error_word, 2);
+                        if (!ok) break;
+                        sh->slot_coeff[s] = sh->batch_coeff[u];
+                        ptx::mbar_arrive_expect_tx(&sh->full[s], STAGE_BYTES);
+                        ptx::bulk_load(ring + (size_t)s * STAGE_BYTES,
+                                       static_cast<const PathT *>(sh->batch_src[u]) + k0, STAGE_BYTES,
+                                       &sh->full[s]);
+                        q.advance(stages);
+                    }
+                }
+                __syncwarp();
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+            }
+            ++t;
+        }
+        // Leave only when every copy this warp started has landed: another CTA may get this
+        // shared memory next.  Waits on already completed phases return at once.
+        if (lane == 0) {
+            for (int back = 0; back < stages && q.used > 0; ++back) {
+                q.retreat(stages);
+                bounded_wait(&sh->full[q.slot], q.phase, p.error_word, 3);
+            }
+            for (unsigned back = 0; back < 2 && back < t; ++back) {
+                const unsigned tt = t - 1 - back;
+                bounded_wait(&sh->io_full[tt & 1], (tt >> 1) & 1, p.error_word, 3);
+            }
+        }
+    } else if (warp == BULK_COMPUTE_WARPS + 1) {
+        // ------------------------------------------------------------------ store warp
+        bool ok = true;
+        while (ok && walk.next(k0)) {
+            const PassDev pass = p.passes[walk.pass];
+            const int b = t & 1;
+            ok = bounded_wait(&sh->out_ready[b], (t >> 1) & 1, p.error_word, 4);
+            if (!ok) break;
+            if (lane == 0) {
+                if (pass.flags & KPASS_UPDATE) {
+                    ptx::bulk_store(p.theta + pass.theta_off + k0, io_tile(b, 0), F32_TILE_BYTES);
+                    ptx::bulk_store(p.momentum + pass.theta_off + k0, io_tile(b, 1), F32_TILE_BYTES);
+                }
+                if (pass.flags & KPASS_PARTIAL_OUT)
+                    ptx::bulk_store(p.partial + pass.partial_off + k0, io_tile(b, 2), F32_TILE_BYTES);
+            }
+            const unsigned char *src = cast_tile(b);
+            for (int j = lane; j < pass.member_count; j += 32) {
+                PathT *dst = static_cast<PathT *>(p.members[pass.member_begin + j]) + k0;
+                ptx::bulk_store(dst, src, STAGE_BYTES);
+            }
+            ptx::bulk_commit();
+            ptx::bulk_wait_read_all();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sh->io_empty[b]);
+            ++t;
+        }
+        ptx::bulk_wait_all();
+    } else {
+        // ------------------------------------------------------------------ compute warps
+        const int ct = threadIdx.x;  // 0 .. BULK_COMPUTE_THREADS-1
+        bool ok = true;
+        while (ok && walk.next(k0)) {
+            const PassDev pass = p.passes[walk.pass];
+            const int b = t & 1;
+            ok = bounded_wait(&sh->io_full[b], (t >> 1) & 1, p.error_word, 5);
+            if (!ok) break;
+            float th[EPT], acc[EPT];
+            float *th_tile = io_tile(b, 0);
+#pragma unroll
+            for (int u = 0; u < NU; ++u) {
+                const int e0 = (u * BULK_COMPUTE_THREADS + ct) * UE;
+#pragma unroll
+                for (int v = 0; v < UE; v += 4) {
+                    const float4 x = *reinterpret_cast<const float4 *>(th_tile + e0 + v);
+                    th[u * UE + v] = x.x; th[u * UE + v + 1] = x.y;
+                    th[u * UE + v + 2] = x.z; th[u * UE + v + 3] = x.w;
+                }
+            }
+            if (pass.flags & KPASS_PARTIAL_IN) {
+                const float *pt = io_tile(b, 2);
+#pragma unroll
+                for (int u = 0; u < NU; ++u) {
+                    const int e0 = (u * BULK_COMPUTE_THREADS + ct) * UE;
+#pragma unroll
+                    for (int v = 0; v < UE; v += 4) {
+                        const float4 x = *reinterpret_cast<const float4 *>(pt + e0 + v);
+                        acc[u * UE + v] = x.x; acc[u * UE + v + 1] = x.y;
+                        acc[u * UE + v + 2] = x.z; acc[u * UE + v + 3] = x.w;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < EPT; ++i) acc[i] = 0.0f;
+            }
+
+            for (int j = 0; j < pass.contrib_count; ++j) {
+                const int s = q.slot;
+                ok = bounded_wait(&sh->full[s], q.phase, p.error_word, 6);
+                if (!ok) break;
+                const float c = sh->slot_coeff[s];
+                const uint4 *slot = reinterpret_cast<const uint4 *>(ring + (size_t)s * STAGE_BYTES);
+                uint4 raw[NU];
+#pragma unroll
+                for (int u = 0; u < NU; ++u) raw[u] = slot[u * BULK_COMPUTE_THREADS + ct];
+#pragma unroll
+                for (int u = 0; u < NU; ++u) {
+                    float x[UE];
+                    Unit<PathT>::widen(raw[u], x);
+#pragma unroll
+                    for (int i = 0; i < UE; ++i)
+                        acc[u * UE + i] = sync_accumulate(acc[u * UE + i], c, th[u * UE + i], x[i]);
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&sh->empty[s]);
+                q.advance(stages);
+            }
+            if (!ok) break;
+
+            if (pass.flags & KPASS_PARTIAL_OUT) {
+                float *pt = io_tile(b, 2);
+#pragma unroll
+                for (int u = 0; u < NU; ++u) {
+                    const int e0 = (u * BULK_COMPUTE_THREADS + ct) * UE;
+#pragma unroll
+                    for (int v = 0; v < UE; v += 4)
+                        *reinterpret_cast<float4 *>(pt + e0 + v) =
+                            make_float4(acc[u * UE + v], acc[u * UE + v + 1], acc[u * UE + v + 2],
+                                        acc[u * UE + v + 3]);
+                }
+            }
+            if (pass.flags & KPASS_UPDATE) {
+                float *mo_tile = io_tile(b, 1);
+#pragma unroll
+                for (int u = 0; u < NU; ++u) {
+                    const int e0 = (u * BULK_COMPUTE_THREADS + ct) * UE;
+#pragma unroll
+                    for (int v = 0; v < UE; v += 4) {
+                        const float4 m4 = *reinterpret_cast<const float4 *>(mo_tile + e0 + v);
+                        const float mo[4] = {m4.x, m4.y, m4.z, m4.w};
+                        float m1[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            sync_nesterov(th[u * UE + v + i], mo[i], acc[u * UE + v + i], p.lr, p.mu,
+                                          th[u * UE + v + i], m1[i]);
+                        *reinterpret_cast<float4 *>(mo_tile + e0 + v) =
+                            make_float4(m1[0], m1[1], m1[2], m1[3]);
+                        *reinterpret_cast<float4 *>(th_tile + e0 + v) =
+                            make_float4(th[u * UE + v], th[u * UE + v + 1], th[u * UE + v + 2],
+                                        th[u * UE + v + 3]);
+                    }
+                }
+            }
+            if (NEED_CAST_TILE && pass.member_count > 0) {
+                uint4 *ct_tile = reinterpret_cast<uint4 *>(cast_tile(b));
+#pragma unroll
+                for (int u = 0; u < NU; ++u)
+                    ct_tile[u * BULK_COMPUTE_THREADS + ct] = Unit<PathT>::narrow(th + u * UE);
+            }
+            ptx::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sh->out_ready[b]);
+            ++t;
+        }
+    }
+}
+
+} // namespace dipaco

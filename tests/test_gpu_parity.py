@@ -1,0 +1,334 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle.
+
+Tolerance (fp32 results theta', m'): |gpu - oracle| <= 1e-6 * (1 + |oracle|).  Path copies must
+equal cast(gpu theta') bit for bit (fp32: the value itself; bf16: round-to-nearest-even) and, for
+bf16, lie within one bf16 ulp of the oracle's copy.  Kernel families, resident and chunked mode
+and repeated runs must agree bitwise.
+"""
+from __future__ import annotations
+
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2403_10616_b200 import binding as B
+from paper_2403_10616_b200 import synth
+from tests import helpers
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def clone_problem(pr):
+    return (pr.theta.clone(), pr.momentum.clone(), [p.clone() for p in pr.paths])
+
+
+def make_ctx(pr, chunk_paths=0, kernel=B.DIPACO_KERNEL_AUTO, weights="cfg"):
+    cfg = pr.cfg
+    code = B.DIPACO_BF16 if cfg.path_dtype == "bf16" else B.DIPACO_F32
+    w = pr.weights if isinstance(weights, str) else weights
+    ctx = B.dipaco_create(cfg.modules_per_level, cfg.level_numel, pr.table, w,
+                          np.float32(cfg.outer_lr), np.float32(cfg.outer_momentum), code,
+                          chunk_paths, 0)
+    B.dipaco_set_kernel(ctx, kernel)
+    return ctx
+
+
+def run_gpu(pr, state, reported="cfg", chunk_paths=0, kernel=B.DIPACO_KERNEL_AUTO, weights="cfg",
+            tuning=None):
+    theta, momentum, paths = state
+    ctx = make_ctx(pr, chunk_paths, kernel, weights)
+    if tuning:
+        B.dipaco_set_tuning(ctx, *tuning)
+    r = pr.reported if isinstance(reported, str) else reported
+    B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths], r)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    launches = B.dipaco_launch_count(ctx)
+    B.dipaco_destroy(ctx)
+    return launches
+
+
+def assert_matches_oracle(pr, before, after, reported="cfg", weights="cfg", threads=8):
+    cfg = pr.cfg
+    th0, mo0, ps0 = before
+    r = pr.reported if isinstance(reported, str) else reported
+    w = pr.weights if isinstance(weights, str) else weights
+    want_th, want_mo, want_ps = helpers.run_oracle(cfg, pr.table, th0, mo0, ps0, w, r,
+                                                   num_threads=threads)
+    got_th = helpers.tensor_to_numpy(after[0])
+    got_mo = helpers.tensor_to_numpy(after[1])
+    for got, want, name in ((got_th, want_th, "theta"), (got_mo, want_mo, "momentum")):
+        err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+        bound = 1e-6 * (1.0 + np.abs(want.astype(np.float64)))
+        assert np.all(err <= bound), "%s max err %g" % (name, float((err / bound).max()))
+    lvl = pr.level_offsets()
+    mod = pr.module_offsets()
+    for i, p in enumerate(after[2]):
+        got = helpers.tensor_to_numpy(p)
+        for l in range(cfg.num_levels):
+            n = cfg.level_numel[l]
+            src = int(mod[l]) + int(pr.table[i, l]) * n
+            slot = got[int(lvl[l]):int(lvl[l]) + n]
+            if cfg.path_dtype == "bf16":
+                np.testing.assert_array_equal(slot, helpers.float_to_bf16_bits_torch(got_th[src:src + n]))
+                ulp = np.abs(slot.astype(np.int32) - want_ps[i][int(lvl[l]):int(lvl[l]) + n].astype(np.int32))
+                assert ulp.max(initial=0) <= 1
+            else:
+                np.testing.assert_array_equal(slot.view(np.uint32), got_th[src:src + n].view(np.uint32))
+
+
+def assert_states_bitwise_equal(a, b):
+    assert torch.equal(a[0].view(torch.int32), b[0].view(torch.int32))
+    assert torch.equal(a[1].view(torch.int32), b[1].view(torch.int32))
+    for x, y in zip(a[2], b[2]):
+        bits = torch.int16 if x.dtype == torch.bfloat16 else torch.int32
+        assert torch.equal(x.view(bits), y.view(bits))
+
+
+def host_state(state):
+    return (helpers.tensor_to_numpy(state[0]), helpers.tensor_to_numpy(state[1]),
+            [helpers.tensor_to_numpy(p) for p in state[2]])
+
+
+# sizes: several tiles plus a ragged tail, all levels 16-byte aligned / deliberately misaligned
+ALIGNED = {3: (3 * 2048 + 72, 2 * 2048 + 8, 5 * 2048 + 1000),
+           5: (3 * 2048 + 72, 2 * 2048 + 8, 2048 + 1000, 4096, 4096 + 16)}
+ODD = {3: (50003, 50003, 50003), 5: (20003, 10001, 10001, 10001, 10001)}
+
+
+@pytest.mark.parametrize("kernel", [B.DIPACO_KERNEL_AUTO, B.DIPACO_KERNEL_VECTOR, B.DIPACO_KERNEL_SCALAR])
+def test_grid2x2_full_parity(kernel):
+    pr = synth.make_problem(synth.CONFIGS["grid2x2"], DEV)
+    before = host_state(clone_problem(pr))
+    state = clone_problem(pr)
+    run_gpu(pr, state, kernel=kernel)
+    assert_matches_oracle(pr, before, state)
+
+
+def test_grid4x4_full_parity_token_weights_and_momentum():
+    pr = synth.make_problem(synth.CONFIGS["grid4x4"], DEV)
+    before = host_state(clone_problem(pr))
+    state = clone_problem(pr)
+    run_gpu(pr, state)
+    assert_matches_oracle(pr, before, state)
+
+
+@pytest.mark.parametrize("name", ["grid16x16", "grid16x16-masked", "grid4x4x4x4"])
+@pytest.mark.parametrize("sizes", ["aligned", "odd"])
+def test_large_grids_scaled_full_parity(name, sizes):
+    base = synth.CONFIGS[name]
+    numel = (ALIGNED if sizes == "aligned" else ODD)[base.num_levels]
+    pr = synth.make_problem(base.scaled(numel), DEV)
+    before = host_state(clone_problem(pr))
+    state = clone_problem(pr)
+    run_gpu(pr, state)
+    assert_matches_oracle(pr, before, state)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_kernel_families_and_tunings_agree_bitwise(dtype):
+    cfg = synth.SyncConfig("mix", (1, 4, 4), (5 * 4096 + 24, 3 * 4096 + 8, 4096 * 2 + 120), dtype,
+                           weights="tokens", momentum_std=1e-4, mask_prob=0.2, seed=5)
+    pr = synth.make_problem(cfg, DEV)
+    ref = clone_problem(pr)
+    run_gpu(pr, ref, kernel=B.DIPACO_KERNEL_SCALAR)
+    for kernel, tuning in [(B.DIPACO_KERNEL_VECTOR, None), (B.DIPACO_KERNEL_AUTO, None),
+                           (B.DIPACO_KERNEL_AUTO, (1, 3, 1)), (B.DIPACO_KERNEL_AUTO, (1, 0, 2)),
+                           (B.DIPACO_KERNEL_AUTO, (2, 2, 1)), (B.DIPACO_KERNEL_AUTO, (1, 0, 4)),
+                           (B.DIPACO_KERNEL_AUTO, (4, 0, 1))]:
+        state = clone_problem(pr)
+        run_gpu(pr, state, kernel=kernel, tuning=tuning)
+        assert_states_bitwise_equal(ref, state)
+
+
+@pytest.mark.parametrize("name", ["grid16x16", "grid16x16-masked", "grid4x4x4x4"])
+def test_chunked_mode_is_bitwise_identical_to_resident(name):
+    base = synth.CONFIGS[name]
+    pr = synth.make_problem(base.scaled(ALIGNED[base.num_levels]), DEV)
+    resident = clone_problem(pr)
+    run_gpu(pr, resident, chunk_paths=0)
+    for chunk in (32, 100):
+        chunked = clone_problem(pr)
+        launches = run_gpu(pr, chunked, chunk_paths=chunk)
+        assert launches > 2
+        assert_states_bitwise_equal(resident, chunked)
+
+
+def test_incremental_api_with_fresh_buffers_for_writeback():
+    base = synth.CONFIGS["grid16x16-masked"]
+    pr = synth.make_problem(base.scaled(ALIGNED[3]), DEV)
+    resident = clone_problem(pr)
+    run_gpu(pr, resident)
+    theta, momentum, paths = clone_problem(pr)
+    ctx = make_ctx(pr, chunk_paths=32)
+    nchunks, scratch = B.dipaco_plan_chunks(ctx)
+    assert nchunks == 8 and scratch > 0
+    B.dipaco_sync_begin(ctx, theta.data_ptr(), momentum.data_ptr(), pr.reported)
+    # out-of-order chunk is refused and changes nothing
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_sync_accumulate(ctx, 1, [p.data_ptr() for p in paths[32:64]])
+    assert e.value.status == B.DIPACO_ESTATE
+    with pytest.raises(B.DipacoError):
+        B.dipaco_sync_writeback(ctx, 0, [p.data_ptr() for p in paths[0:32]])
+    for c in range(nchunks):
+        # each chunk is staged through the same device buffer, as a streaming caller would
+        stage = [p.clone() for p in paths[32 * c:32 * c + 32]]
+        B.dipaco_sync_accumulate(ctx, c, [p.data_ptr() for p in stage])
+        torch.cuda.synchronize()
+    out_paths = []
+    for c in range(nchunks):
+        fresh = [torch.full_like(p, float("nan")) for p in paths[32 * c:32 * c + 32]]
+        B.dipaco_sync_writeback(ctx, c, [p.data_ptr() for p in fresh])
+        out_paths.extend(fresh)
+    B.dipaco_sync_end(ctx)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    B.dipaco_destroy(ctx)
+    assert_states_bitwise_equal((theta, momentum, out_paths), resident)
+
+
+def test_forced_empty_module_and_all_masked_call():
+    base = synth.CONFIGS["grid16x16-masked"]
+    pr = synth.make_problem(base.scaled(ALIGNED[3]), DEV)
+    reported = pr.reported.copy()
+    reported[[i for i in range(256) if pr.table[i, 1] == 3]] = 0   # level-1 module 3 loses everyone
+    for chunk in (0, 32):
+        before = host_state(clone_problem(pr))
+        state = clone_problem(pr)
+        run_gpu(pr, state, reported=reported, chunk_paths=chunk)
+        assert_matches_oracle(pr, before, state, reported=reported)
+        n0, n1, _ = pr.cfg.level_numel
+        sl = slice(n0 + 3 * n1, n0 + 4 * n1)
+        assert torch.equal(state[0][sl].view(torch.int32), pr.theta[sl].view(torch.int32))
+        assert torch.equal(state[1][sl].view(torch.int32), pr.momentum[sl].view(torch.int32))
+    none = np.zeros(256, dtype=np.uint8)
+    state = clone_problem(pr)
+    run_gpu(pr, state, reported=none)
+    assert torch.equal(state[0].view(torch.int32), pr.theta.view(torch.int32))
+    assert torch.equal(state[1].view(torch.int32), pr.momentum.view(torch.int32))
+    before = host_state(clone_problem(pr))
+    assert_matches_oracle(pr, before, state, reported=none)
+
+
+def test_masked_paths_are_not_read_and_nan_propagates():
+    cfg = synth.CONFIGS["grid4x4"].scaled((4096 + 8, 2048 + 16, 2048))
+    pr = synth.make_problem(cfg, DEV)
+    reported = np.ones(16, dtype=np.uint8)
+    reported[5] = 0
+    clean = clone_problem(pr)
+    run_gpu(pr, clean, reported=reported)
+    dirty = clone_problem(pr)
+    dirty[2][5].fill_(float("nan"))
+    run_gpu(pr, dirty, reported=reported)
+    assert_states_bitwise_equal(clean, dirty)
+    # a NaN in a reporting copy reaches exactly the elements it touches
+    state = clone_problem(pr)
+    state[2][2][7] = float("nan")
+    run_gpu(pr, state, reported=reported)
+    assert torch.isnan(state[0][7]) and not torch.isnan(state[0][8])
+    assert torch.isnan(state[0]).sum().item() == 1
+
+
+def test_misaligned_path_pointers_take_the_scalar_path():
+    cfg = synth.SyncConfig("mis", (1, 2, 2), (4100, 2052, 1000), "bf16", seed=9)
+    pr = synth.make_problem(cfg, DEV)
+    before = host_state(clone_problem(pr))
+    per = cfg.params_per_path
+    backing = [torch.empty(per + 8, dtype=torch.bfloat16, device=DEV) for _ in range(4)]
+    paths = []
+    for i, b in enumerate(backing):
+        view = b[1 + i:1 + i + per]          # 2-byte aligned only
+        view.copy_(pr.paths[i])
+        paths.append(view)
+    state = (pr.theta.clone(), pr.momentum.clone(), paths)
+    run_gpu(pr, state)
+    assert_matches_oracle(pr, before, state)
+
+
+def test_runs_are_bitwise_reproducible():
+    base = synth.CONFIGS["grid4x4x4x4"]
+    cfg = base.scaled((20 * 2048 + 8, 10 * 2048, 10 * 2048 + 16, 10 * 2048, 10 * 2048 + 1000))
+    results = []
+    for _ in range(3):
+        pr = synth.make_problem(cfg, DEV)       # regenerated from the seed every time
+        state = (pr.theta, pr.momentum, pr.paths)
+        run_gpu(pr, state)
+        results.append(state)
+    assert_states_bitwise_equal(results[0], results[1])
+    assert_states_bitwise_equal(results[0], results[2])
+
+
+def test_two_rounds_on_one_context_follow_the_oracle():
+    cfg = synth.CONFIGS["grid4x4"].scaled((3 * 2048 + 24, 2048 + 8, 2048 + 40))
+    pr = synth.make_problem(cfg, DEV)
+    th, mo, ps = host_state(clone_problem(pr))
+    theta, momentum, paths = clone_problem(pr)
+    ctx = make_ctx(pr)
+    rng = np.random.RandomState(3)
+    for rnd in range(2):
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths],
+                            pr.reported)
+        th, mo, ps = helpers.run_oracle(cfg, pr.table, th, mo, ps, pr.weights, pr.reported)
+        err = np.abs(helpers.tensor_to_numpy(theta).astype(np.float64) - th)
+        assert np.all(err <= 1e-6 * (1 + np.abs(th)))
+        # next inner phase: every path drifts away from the synchronised value again
+        for i in range(cfg.num_paths):
+            drift = rng.normal(0, 1e-3, cfg.params_per_path).astype(np.float32)
+            ps[i] = ps[i] + drift
+            paths[i].copy_(torch.from_numpy(ps[i]))
+        # keep the oracle's global state equal to the device's so errors do not compound
+        th = helpers.tensor_to_numpy(theta)
+        mo = helpers.tensor_to_numpy(momentum)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    assert B.dipaco_launch_count(ctx) >= 2
+    B.dipaco_destroy(ctx)
+
+
+def test_argument_errors_leave_buffers_untouched():
+    pr = synth.make_problem(synth.CONFIGS["grid2x2"], DEV)
+    state = clone_problem(pr)
+    ctx = make_ctx(pr)
+    ptrs = [p.data_ptr() for p in state[2]]
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_outer_sync(ctx, 0, state[1].data_ptr(), ptrs)
+    assert e.value.status == B.DIPACO_EINVAL
+    with pytest.raises(B.DipacoError):
+        B.dipaco_outer_sync(ctx, state[0].data_ptr(), state[1].data_ptr(), ptrs[:3] + [0])
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_sync_begin(ctx, state[0].data_ptr(), state[1].data_ptr())   # not a chunked context
+    assert e.value.status == B.DIPACO_ESTATE
+    torch.cuda.synchronize()
+    assert_states_bitwise_equal(state, clone_problem(pr))
+    B.dipaco_destroy(ctx)
+
+
+@pytest.mark.parametrize("name,pinned", [("grid16x16-masked", True), ("grid4x4", False)])
+def test_host_buffers_entry_point_matches_the_oracle(name, pinned):
+    base = synth.CONFIGS[name]
+    numel = ALIGNED[3] if name != "grid4x4" else (3 * 2048 + 24, 2048 + 8, 50003)
+    cfg = base.scaled(numel)
+    pr = synth.make_problem(cfg, "cpu")
+    before = host_state(clone_problem(pr))
+    theta, momentum, paths = clone_problem(pr)
+    if pinned:
+        theta, momentum = theta.pin_memory(), momentum.pin_memory()
+        paths = [p.pin_memory() for p in paths]
+    chunk = 32 if cfg.num_paths > 32 else 5
+    ctx = make_ctx(pr, chunk_paths=chunk)
+    for rnd in range(2):            # second call reuses the staging buffers
+        if rnd == 1:
+            theta.copy_(pr.theta); momentum.copy_(pr.momentum)
+            for p, q in zip(paths, pr.paths):
+                p.copy_(q)
+        B.dipaco_outer_sync_host(ctx, theta.data_ptr(), momentum.data_ptr(),
+                                 [p.data_ptr() for p in paths], pr.reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        assert_matches_oracle(pr, before, (theta, momentum, paths))
+    B.dipaco_destroy(ctx)
+    # and it is bitwise the device-resident result
+    dev = synth.make_problem(cfg, "cpu")
+    state = (dev.theta.to(DEV), dev.momentum.to(DEV), [p.to(DEV) for p in dev.paths])
+    run_gpu(pr, state)
+    assert_states_bitwise_equal((theta.to(DEV), momentum.to(DEV), [p.to(DEV) for p in paths]), state)

@@ -1,0 +1,216 @@
+"""CPU tests of the CUDA library's host side: exported symbols, validation, planning (step a0).
+
+No compute call is made: contexts are created plan-only (device = -1)."""
+from __future__ import annotations
+
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2403_10616_b200 import binding as B
+from paper_2403_10616_b200 import build as libbuild
+from paper_2403_10616_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built_library():
+    libbuild.build()
+    B.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "dipaco.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dipaco_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(B.LIB_PATH)
+    names = declared_functions()
+    assert "dipaco_create" in names and "dipaco_outer_sync" in names and "dipaco_destroy" in names
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(B.EXPORTS) == names
+
+
+def test_strerror_names_every_status():
+    for code in (0, -1, -2, -3, -4, -5, -6):
+        assert B.strerror(code) != "unknown status"
+    assert B.strerror(-99) == "unknown status"
+
+
+def plan_ctx(cfg, table=None, weights=None, chunk_paths=0):
+    table = synth.path_table(cfg.modules_per_level) if table is None else table
+    code = B.DIPACO_BF16 if cfg.path_dtype == "bf16" else B.DIPACO_F32
+    return B.dipaco_create(cfg.modules_per_level, cfg.level_numel, table, weights,
+                           cfg.outer_lr, cfg.outer_momentum, code, chunk_paths, device=-1)
+
+
+def test_plan_only_context_refuses_compute_calls():
+    cfg = synth.CONFIGS["grid2x2"]
+    ctx = plan_ctx(cfg)
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_outer_sync(ctx, 16, 16, [16] * cfg.num_paths, None, stream=0)
+    assert e.value.status == B.DIPACO_ENODEV
+    assert B.dipaco_device_status(ctx) == B.DIPACO_ENODEV
+    B.dipaco_destroy(ctx)
+
+
+@pytest.mark.parametrize("bad", ["entry", "negative_entry", "levels", "weights_nan", "weights_neg",
+                                 "k_zero", "n_negative", "lr_inf", "dtype"])
+def test_create_rejects_invalid_arguments(bad):
+    K = np.array([1, 2, 2], dtype=np.int32)
+    N = np.array([8, 8, 8], dtype=np.int64)
+    table = synth.path_table(K).copy()
+    w = np.ones(4, dtype=np.float32)
+    lr, dtype = 0.7, B.DIPACO_F32
+    if bad == "entry":
+        table[2, 1] = 2
+    elif bad == "negative_entry":
+        table[0, 0] = -1
+    elif bad == "weights_nan":
+        w[1] = np.nan
+    elif bad == "weights_neg":
+        w[1] = -1.0
+    elif bad == "k_zero":
+        K[2] = 0
+    elif bad == "n_negative":
+        N[0] = -5
+    elif bad == "lr_inf":
+        lr = float("inf")
+    elif bad == "dtype":
+        dtype = 7
+    if bad == "levels":
+        lib = B.load()
+        h = ctypes.c_void_p()
+        rc = lib.dipaco_create(ctypes.byref(h), 0, K.ctypes.data, N.ctypes.data, 4, table.ctypes.data,
+                               None, 0.7, 0.9, 0, 0, -1)
+        assert rc == B.DIPACO_EINVAL and not h.value
+        return
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_create(K, N, table, w, lr, 0.9, dtype, 0, device=-1)
+    assert e.value.status == B.DIPACO_EINVAL
+
+
+def test_toy_grid_contributor_sets_match_the_papers_figure():
+    cfg = synth.CONFIGS["grid2x2"]
+    ctx = plan_ctx(cfg)
+    want = {(0, 0): [0, 1, 2, 3], (1, 0): [0, 1], (1, 1): [2, 3], (2, 0): [0, 2], (2, 1): [1, 3]}
+    for (l, e), paths in want.items():
+        members, contributors, coeff, upd = B.dipaco_plan_module(ctx, l, e, cfg.num_paths)
+        assert members.tolist() == paths and contributors.tolist() == paths and upd
+        np.testing.assert_array_equal(coeff, np.full(len(paths), 1.0 / len(paths), np.float32))
+    B.dipaco_destroy(ctx)
+
+
+def test_coefficients_are_normalised_per_module_over_reporting_paths():
+    cfg = synth.CONFIGS["grid16x16-masked"].scaled((16, 16, 16))
+    w = synth.path_weights(cfg)
+    r = synth.reported_mask(cfg)
+    table = synth.path_table(cfg.modules_per_level)
+    ctx = plan_ctx(cfg, table, w)
+    for l in range(3):
+        for e in range(cfg.modules_per_level[l]):
+            members, contributors, coeff, upd = B.dipaco_plan_module(ctx, l, e, cfg.num_paths, r)
+            S = [i for i in range(cfg.num_paths) if table[i, l] == e]
+            R = [i for i in S if r[i]]
+            assert members.tolist() == S and contributors.tolist() == R and upd
+            total = np.sum(w[R].astype(np.float64))
+            np.testing.assert_array_equal(coeff, (w[R].astype(np.float64) / total).astype(np.float32))
+            assert abs(float(np.sum(coeff.astype(np.float64))) - 1.0) < 1e-6
+    # a module whose paths are all masked, and zero total weight
+    r2 = r.copy()
+    r2[[i for i in range(cfg.num_paths) if table[i, 1] == 3]] = 0
+    members, contributors, coeff, upd = B.dipaco_plan_module(ctx, 1, 3, cfg.num_paths, r2)
+    assert len(members) == 16 and len(contributors) == 0 and not upd
+    w0 = w.copy()
+    w0[[i for i in range(cfg.num_paths) if table[i, 2] == 5]] = 0.0
+    B.dipaco_set_weights(ctx, w0)
+    _, contributors, _, upd = B.dipaco_plan_module(ctx, 2, 5, cfg.num_paths, None)
+    assert len(contributors) == 0 and not upd
+    B.dipaco_set_weights(ctx, None)
+    _, contributors, coeff, upd = B.dipaco_plan_module(ctx, 2, 5, cfg.num_paths, None)
+    assert upd and np.all(coeff == np.float32(1 / 16))
+    B.dipaco_destroy(ctx)
+
+
+def test_offsets_follow_level_module_element_order():
+    cfg = synth.CONFIGS["grid4x4x4x4"].scaled((7, 5, 3, 11, 2))
+    ctx = plan_ctx(cfg)
+    theta_off = 0
+    path_off = 0
+    for l, (k, n) in enumerate(zip(cfg.modules_per_level, cfg.level_numel)):
+        for e in range(k):
+            assert B.dipaco_plan_offsets(ctx, l, e) == (theta_off, path_off, n)
+            theta_off += n
+        path_off += n
+    with pytest.raises(B.DipacoError):
+        B.dipaco_plan_offsets(ctx, 1, 4)
+    B.dipaco_destroy(ctx)
+
+
+def test_arbitrary_subset_of_paths_and_unused_modules():
+    """Any path set is allowed (path sampling); a module nobody uses has no members."""
+    K, N = (1, 3, 3), (4, 4, 4)
+    table = np.array([[0, 0, 1], [0, 2, 1], [0, 2, 2]], dtype=np.int32)
+    ctx = B.dipaco_create(K, N, table, None, 0.7, 0.9, B.DIPACO_F32, 0, device=-1)
+    members, contributors, _, upd = B.dipaco_plan_module(ctx, 1, 1, 3)
+    assert len(members) == 0 and len(contributors) == 0 and not upd
+    members, _, coeff, _ = B.dipaco_plan_module(ctx, 1, 2, 3)
+    assert members.tolist() == [1, 2] and coeff.tolist() == [0.5, 0.5]
+    B.dipaco_destroy(ctx)
+
+
+def test_chunk_count_and_scratch_size():
+    cfg = synth.CONFIGS["grid16x16"].scaled((1000, 1001, 1002))
+    ctx = plan_ctx(cfg, chunk_paths=32)
+    n, scratch = B.dipaco_plan_chunks(ctx)
+    # shared level and the 16 level-2 modules span chunks; level-1 modules live inside one chunk
+    assert n == 8 and scratch == 1000 + 16 * 1004
+    B.dipaco_destroy(ctx)
+    ctx = plan_ctx(cfg, chunk_paths=0)
+    assert B.dipaco_plan_chunks(ctx) == (1, 0)
+    B.dipaco_destroy(ctx)
+    ctx = plan_ctx(cfg, chunk_paths=100)
+    assert B.dipaco_plan_chunks(ctx)[0] == 3
+    B.dipaco_destroy(ctx)
+
+
+@pytest.mark.parametrize("name,numel,ctas", [("grid16x16", (50_000_000,) * 3, 296),
+                                             ("grid4x4x4x4", (20_000_000,) + (10_000_000,) * 4, 148),
+                                             ("grid2x2", (16384, 65536, 65536), 296),
+                                             ("grid4x4", (4096 + 17, 2048 * 3, 100), 7)])
+def test_split_covers_every_full_tile_once_and_balances_cost(name, numel, ctas):
+    cfg = synth.CONFIGS[name].scaled(numel)
+    tile = 2048
+    ctx = plan_ctx(cfg)
+    lvl, mod, beg, end, first = B.dipaco_plan_split(ctx, ctas, tile)
+    assert first[0] == 0 and first[-1] == len(lvl) and np.all(np.diff(first) >= 0)
+    assert np.all(beg % tile == 0) and np.all(end % tile == 0) and np.all(end > beg)
+    covered = {}
+    for l, e, b, t in zip(lvl, mod, beg, end):
+        covered.setdefault((int(l), int(e)), []).append((int(b), int(t)))
+    for l, (k, n) in enumerate(zip(cfg.modules_per_level, cfg.level_numel)):
+        full = n // tile * tile
+        for e in range(k):
+            spans = sorted(covered.get((l, e), []))
+            pos = 0
+            for b, t in spans:
+                assert b == pos
+                pos = t
+            assert pos == full
+    # bytes per element: theta r/w + momentum r/w + contributors read + members written
+    s = 2 if cfg.path_dtype == "bf16" else 4
+    per_level = [16 + 2 * s * (cfg.num_paths // k) for k in cfg.modules_per_level]
+    cost = np.zeros(ctas)
+    for b in range(ctas):
+        for i in range(first[b], first[b + 1]):
+            cost[b] += per_level[lvl[i]] * (end[i] - beg[i])
+    heaviest_tile = max(per_level) * tile
+    assert cost.max() - cost.sum() / ctas <= 1.01 * heaviest_tile
+    B.dipaco_destroy(ctx)
