@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 METRIC = "outer_sync_path_params_per_s"
 UNIT = "path-params/s"
-CPU_SAMPLE_NUMEL = 4_000_000      # parameters per level in the CPU-baseline sample
+CPU_SAMPLE_NUMEL = 10_000_000     # parameters per level in the CPU-baseline sample
 REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the reference arm
 
 

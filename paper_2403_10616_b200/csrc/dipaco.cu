@@ -123,7 +123,7 @@ size_t bulk_smem_bytes(const dipaco_ctx *ctx, int stages, int io_arrays)
 int pick_stages(const dipaco_ctx *ctx, int io_arrays)
 {
     const size_t budget =
-        std::min(SMEM_LIMIT, SMEM_PER_SM / (size_t)ctx->ctas_per_sm - SMEM_CTA_RESERVE);
+        std::min(SMEM_LIMIT, SMEM_PER_SM / (size_t)ctx->ctas_per_sm - 2 * SMEM_CTA_RESERVE);
     int best = 0;
     for (int s = 2; s <= BULK_MAX_STAGES; ++s)
         if (bulk_smem_bytes(ctx, s, io_arrays) <= budget) best = s;
@@ -520,7 +520,9 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
     if (ctas_per_sm) ctx->ctas_per_sm = ctas_per_sm;
     if (units_per_thread) ctx->units = units_per_thread;
     ctx->stages = 0;
-    const bool fits = pick_stages(ctx, 3) >= 2 && (!stages || stages <= pick_stages(ctx, 2));
+    // chunked contexts stage a third fp32 tile (the partial sum) per buffer
+    const int io_arrays = ctx->grid.num_chunks > 1 ? 3 : 2;
+    const bool fits = pick_stages(ctx, io_arrays) >= 2 && (!stages || stages <= pick_stages(ctx, io_arrays));
     if (!fits) {
         ctx->ctas_per_sm = old_ctas;
         ctx->units = old_units;

@@ -2,7 +2,7 @@
 
 Tolerance (fp32 results theta', m'): |gpu - oracle| <= 1e-6 * (1 + |oracle|).  Path copies must
 equal cast(gpu theta') bit for bit (fp32: the value itself; bf16: round-to-nearest-even) and, for
-bf16, lie within one bf16 ulp of the oracle's copy.  Kernel families, resident and chunked mode
+bf16, lie within one bf16 rounding step plus the fp32 tolerance of the oracle's copy.  Kernel families, resident and chunked mode
 and repeated runs must agree bitwise.
 """
 from __future__ import annotations
@@ -74,10 +74,18 @@ def assert_matches_oracle(pr, before, after, reported="cfg", weights="cfg", thre
             slot = got[int(lvl[l]):int(lvl[l]) + n]
             if cfg.path_dtype == "bf16":
                 np.testing.assert_array_equal(slot, helpers.float_to_bf16_bits_torch(got_th[src:src + n]))
-                ulp = np.abs(slot.astype(np.int32) - want_ps[i][int(lvl[l]):int(lvl[l]) + n].astype(np.int32))
-                assert ulp.max(initial=0) <= 1
+                assert_bf16_close(slot, want_ps[i][int(lvl[l]):int(lvl[l]) + n])
             else:
                 np.testing.assert_array_equal(slot.view(np.uint32), got_th[src:src + n].view(np.uint32))
+
+
+def assert_bf16_close(got_bits, want_bits):
+    """Two roundings of nearly equal fp32 values: at most one bf16 step (2^-7 relative) on top of
+    the fp32 tolerance (which dominates where theta' is close to zero)."""
+    got = helpers.bf16_bits_to_float(got_bits).astype(np.float64)
+    want = helpers.bf16_bits_to_float(want_bits).astype(np.float64)
+    bound = 1e-6 * (1.0 + np.abs(want)) + 2.0 ** -7 * np.abs(want)
+    assert np.all(np.abs(got - want) <= bound)
 
 
 def assert_states_bitwise_equal(a, b):
@@ -138,7 +146,7 @@ def test_kernel_families_and_tunings_agree_bitwise(dtype):
     for kernel, tuning in [(B.DIPACO_KERNEL_VECTOR, None), (B.DIPACO_KERNEL_AUTO, None),
                            (B.DIPACO_KERNEL_AUTO, (1, 3, 1)), (B.DIPACO_KERNEL_AUTO, (1, 0, 2)),
                            (B.DIPACO_KERNEL_AUTO, (2, 2, 1)), (B.DIPACO_KERNEL_AUTO, (1, 0, 4)),
-                           (B.DIPACO_KERNEL_AUTO, (4, 0, 1))]:
+                           (B.DIPACO_KERNEL_AUTO, (3, 0, 1))]:
         state = clone_problem(pr)
         run_gpu(pr, state, kernel=kernel, tuning=tuning)
         assert_states_bitwise_equal(ref, state)
