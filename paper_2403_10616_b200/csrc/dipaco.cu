@@ -20,6 +20,8 @@ constexpr size_t SMEM_LIMIT = 227 * 1024;  // opt-in dynamic shared memory per C
 constexpr size_t SMEM_PER_SM = 228 * 1024;
 constexpr size_t SMEM_CTA_RESERVE = 1024;  // per-CTA reservation the driver adds
 constexpr int64_t RAGGED_TILE = 1024;      // split granularity of the scalar kernel
+constexpr int MAX_COUNTERS = 256;          // work counters (one per bulk launch of an upload)
+constexpr double ITEM_TARGET_BYTES = 2.0 * 1024 * 1024;  // traffic of one dynamic work item
 
 enum SyncState { STATE_IDLE = 0, STATE_ACCUMULATING = 1 };
 
@@ -37,6 +39,7 @@ struct PackedLaunch {
     int bulk_ctas = 0, rag_ctas = 0;
     int io_arrays = 2;
     bool aligned_kernel_is_vector = false;
+    int num_passes = 0, total_items = 0;  // dynamic scheduling of the bulk-copy kernel
 };
 
 struct HostMode;  // state of dipaco_outer_sync_host (host_mode.inl)
@@ -51,7 +54,7 @@ struct dipaco_ctx {
     int device = -1;
     int sm_count = 0;
     int kernel = DIPACO_KERNEL_AUTO;
-    int ctas_per_sm = 2, stages = 0, units = 0;  // 0 = automatic
+    int ctas_per_sm = 1, stages = 10, units = 2;  // bulk-copy kernel tuning (measured on B200)
     int64_t launches = 0;
 
     void *dev_tables = nullptr;
@@ -60,6 +63,7 @@ struct dipaco_ctx {
     int staging_next = 0;
     float *partial = nullptr;
     int *error_word = nullptr;
+    int *counters = nullptr;  // MAX_COUNTERS work counters for the bulk-copy kernel
     bool smem_attr_set[2][3] = {{false, false, false}, {false, false, false}};
 
     // round state of the incremental API
@@ -100,8 +104,7 @@ void compute_all_coeffs(dipaco_ctx *ctx, const uint8_t *reported)
 
 int tile_units(const dipaco_ctx *ctx)
 {
-    if (ctx->units > 0) return ctx->units;
-    return ctx->dtype == DIPACO_BF16 ? 1 : 2;
+    return ctx->units > 0 ? ctx->units : 2;
 }
 
 int64_t tile_elems(const dipaco_ctx *ctx)
@@ -168,6 +171,9 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         pd.partial_off = m.partial_off >= 0 ? m.partial_off : 0;
         pd.flags = sp.flags;
         pd.pad = 0;
+        pd.item_first = 0;
+        pd.tiles_per_item = 1;
+        pd.bulk_tiles = 0;
         if ((sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) && (m.partial_off < 0 || !ctx->partial))
             return DIPACO_ESTATE;
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
@@ -211,14 +217,34 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     const bool vector_kernel = ctx->kernel == DIPACO_KERNEL_VECTOR;
     int bulk_ctas = ctx->sm_count * (vector_kernel ? 8 : ctx->ctas_per_sm);
     int64_t bulk_tiles = 0, rag_tiles = 0;
+    double bulk_bytes = 0.0;
     for (size_t i = 0; i < specs.size(); ++i) {
         bulk_tiles += (bulk_end[i] - bulk_begin[i]) / tile;
+        bulk_bytes += pass_cost_per_elem(specs[i], es) * (double)(bulk_end[i] - bulk_begin[i]);
         rag_tiles += (rag_end[i] - rag_begin[i] + RAGGED_TILE - 1) / RAGGED_TILE;
     }
     if (bulk_tiles < bulk_ctas) bulk_ctas = (int)bulk_tiles;
     int rag_ctas = (int)std::min<int64_t>(rag_tiles, (int64_t)ctx->sm_count * 8);
-    if (bulk_ctas > 0)
+    int64_t total_items = 0;
+    if (bulk_ctas > 0 && vector_kernel) {
         split_segments(specs, bulk_begin, bulk_end, es, tile, bulk_ctas, bulk_segs, bulk_first);
+    } else if (bulk_ctas > 0) {
+        // Work items of about equal traffic, small enough that every CTA draws many of them.
+        const double target = std::min(ITEM_TARGET_BYTES, bulk_bytes / ((double)bulk_ctas * 16.0));
+        for (size_t i = 0; i < specs.size(); ++i) {
+            const int64_t ntiles = (bulk_end[i] - bulk_begin[i]) / tile;
+            const double per_tile = pass_cost_per_elem(specs[i], es) * (double)tile;
+            int64_t tpi = (int64_t)std::floor(target / per_tile + 0.5);
+            if (tpi < 1) tpi = 1;
+            if (tpi > (1 << 20)) tpi = 1 << 20;
+            passes[i].item_first = (int)total_items;
+            passes[i].tiles_per_item = (int)tpi;
+            passes[i].bulk_tiles = ntiles;
+            total_items += (ntiles + tpi - 1) / tpi;
+        }
+        if (total_items > 0x7fff0000) return DIPACO_EINVAL;
+        if (total_items < bulk_ctas) bulk_ctas = (int)total_items;
+    }
     if (rag_ctas > 0)
         split_segments(specs, rag_begin, rag_end, es, RAGGED_TILE, rag_ctas, rag_segs, rag_first);
 
@@ -240,6 +266,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     out.rag_ctas = rag_ctas;
     out.io_arrays = any_partial ? 3 : 2;
     out.aligned_kernel_is_vector = vector_kernel;
+    out.num_passes = (int)passes.size();
+    out.total_items = (int)total_items;
     return DIPACO_OK;
 }
 
@@ -319,7 +347,7 @@ int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays
 }
 
 int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *momentum,
-                  cudaStream_t stream)
+                  int *work_counter, cudaStream_t stream)
 {
     const char *base = static_cast<const char *>(ctx->dev_tables);
     LaunchParams lp;
@@ -332,6 +360,9 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
     lp.lr = ctx->lr;
     lp.mu = ctx->mu;
     lp.error_word = ctx->error_word;
+    lp.num_passes = pl.num_passes;
+    lp.total_items = pl.total_items;
+    lp.work_counter = work_counter;
     if (pl.bulk_ctas > 0) {
         lp.segs = reinterpret_cast<const SegmentDev *>(base + pl.bulk_segs_off);
         lp.cta_first = reinterpret_cast<const int *>(base + pl.bulk_first_off);
@@ -382,7 +413,13 @@ int run_launches(dipaco_ctx *ctx, std::vector<LaunchRequest> &reqs, float *theta
     int rc = upload_blob(ctx, blob, stream);
     if (rc != DIPACO_OK) return rc;
     for (size_t i = 0; i < reqs.size(); ++i) {
-        rc = launch_packed(ctx, packed[i], theta, momentum, stream);
+        const int c = (int)(i % MAX_COUNTERS);
+        if (c == 0) {
+            const size_t n = std::min<size_t>(MAX_COUNTERS, reqs.size() - i);
+            if (cudaMemsetAsync(ctx->counters, 0, n * sizeof(int), stream) != cudaSuccess)
+                return DIPACO_ECUDA;
+        }
+        rc = launch_packed(ctx, packed[i], theta, momentum, ctx->counters + c, stream);
         if (rc != DIPACO_OK) return rc;
     }
     ctx->last_stream = stream;
@@ -448,7 +485,8 @@ int dipaco_create(dipaco_ctx **out, int32_t num_levels, const int32_t *modules_p
             return DIPACO_ECUDA;
         }
         if (cudaMalloc(&ctx->error_word, sizeof(int)) != cudaSuccess ||
-            cudaMemset(ctx->error_word, 0, sizeof(int)) != cudaSuccess) {
+            cudaMemset(ctx->error_word, 0, sizeof(int)) != cudaSuccess ||
+            cudaMalloc(&ctx->counters, MAX_COUNTERS * sizeof(int)) != cudaSuccess) {
             dipaco_destroy(ctx);
             return DIPACO_ENOMEM;
         }
@@ -481,6 +519,7 @@ int dipaco_destroy(dipaco_ctx *ctx)
         if (ctx->dev_tables) cudaFree(ctx->dev_tables);
         if (ctx->partial) cudaFree(ctx->partial);
         if (ctx->error_word) cudaFree(ctx->error_word);
+        if (ctx->counters) cudaFree(ctx->counters);
     }
     delete ctx;
     return rc;

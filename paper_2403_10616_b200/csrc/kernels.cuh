@@ -23,7 +23,13 @@ struct PassDev {
     long long partial_off;  // elements into the partial-sum scratch (valid with PARTIAL flags)
     int contrib_begin, contrib_count;
     int member_begin, member_count;
-    int flags, pad;
+    int flags;
+    // dynamic scheduling of the bulk-copy kernel: this pass owns work items
+    // [item_first, item_first + ceil(bulk_tiles / tiles_per_item)), each a run of full tiles
+    int item_first;
+    int tiles_per_item;
+    int pad;
+    long long bulk_tiles;
 };
 
 struct ContribDev {
@@ -48,6 +54,10 @@ struct LaunchParams {
     const int *cta_first;  // [gridDim.x + 1]
     float lr, mu;
     int *error_word;
+    // bulk-copy kernel only
+    int num_passes;
+    int total_items;
+    int *work_counter;  // zeroed before the launch; CTAs draw work items from it
 };
 
 // ------------------------------------------------------------------------------------------
@@ -339,8 +349,10 @@ __device__ __forceinline__ void fence_proxy_async()
 
 constexpr int BULK_COMPUTE_WARPS = 8;
 constexpr int BULK_COMPUTE_THREADS = BULK_COMPUTE_WARPS * 32;
-constexpr int BULK_THREADS = BULK_COMPUTE_THREADS + 64;  // + load warp + store warp
+constexpr int BULK_THREADS = BULK_COMPUTE_THREADS + 96;  // + load, store and scheduler warps
 constexpr int BULK_MAX_STAGES = 32;
+constexpr int BULK_SCHED_DEPTH = 4;
+constexpr int BULK_ITEM_READERS = BULK_COMPUTE_WARPS + 2;  // warps that consume every work item
 constexpr unsigned long long BULK_WAIT_LIMIT_NS = 4000000000ull;  // every wait gives up after 4 s
 
 // Bounded wait: returns false (and records the failure) if the phase does not complete in time.
@@ -365,6 +377,10 @@ struct BulkShared {
     uint64_t io_full[2];              // theta / momentum / partial tiles loaded
     uint64_t io_empty[2];             // result tiles drained by the store warp
     uint64_t out_ready[2];            // compute warps finished writing the result tiles
+    uint64_t sched_full[BULK_SCHED_DEPTH];   // a work item was published by the scheduler warp
+    uint64_t sched_empty[BULK_SCHED_DEPTH];  // all ten consumer warps have read it
+    long long sched_begin[BULK_SCHED_DEPTH], sched_end[BULK_SCHED_DEPTH];
+    int sched_pass[BULK_SCHED_DEPTH];        // -1 = no more work
     float slot_coeff[BULK_MAX_STAGES];
     const void *batch_src[32];
     float batch_coeff[32];
@@ -387,27 +403,38 @@ struct RingPos {
     }
 };
 
-// Tile walk shared by the three roles: every role visits the same (pass, first element) sequence.
-struct TileWalk {
-    const SegmentDev *segs;
-    int seg, seg_end;
-    long long pos, end;
-    int pass;
+// Work items are drawn from a global counter by the scheduler warp and published through a
+// small shared-memory ring; the load, store and compute warps all walk the same item sequence.
+struct ItemWalk {
+    BulkShared *sh;
+    int *error_word;
     long long tile;
-    __device__ TileWalk(const LaunchParams &p, long long tile_elems)
-        : segs(p.segs), seg(p.cta_first[blockIdx.x]), seg_end(p.cta_first[blockIdx.x + 1]), pos(0),
-          end(0), pass(-1), tile(tile_elems)
+    int lane;
+    int slot = 0;
+    unsigned phase = 0;
+    int pass = -1;
+    long long pos = 0, end = 0;
+    __device__ ItemWalk(BulkShared *shared, int *err, long long tile_elems, int lane_id)
+        : sh(shared), error_word(err), tile(tile_elems), lane(lane_id)
     {
-        seg -= 1;
     }
-    __device__ bool next(long long &k0)
+    // Next tile of this CTA: sets pass and k0; false when the work is exhausted (ok stays true)
+    // or a wait ran out (ok = false).  Must be called by all lanes of the warp together.
+    __device__ bool next(long long &k0, bool &ok)
     {
-        if (pass >= 0) pos += tile;
-        while (pass < 0 || pos >= end) {
-            if (++seg >= seg_end) return false;
-            const SegmentDev s = segs[seg];
-            pass = s.pass; pos = s.begin; end = s.end;
+        if (pass >= 0) {
+            pos += tile;
+            if (pos < end) { k0 = pos; return true; }
         }
+        ok = bounded_wait(&sh->sched_full[slot], phase, error_word, 7);
+        if (!ok) return false;
+        const int item_pass = sh->sched_pass[slot];
+        const long long b = sh->sched_begin[slot], e = sh->sched_end[slot];
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&sh->sched_empty[slot]);
+        if (++slot == BULK_SCHED_DEPTH) { slot = 0; phase ^= 1u; }
+        if (item_pass < 0) return false;
+        pass = item_pass; pos = b; end = e;
         k0 = pos;
         return true;
     }
@@ -440,6 +467,10 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
             ptx::mbar_init(&sh->full[s], 1);
             ptx::mbar_init(&sh->empty[s], BULK_COMPUTE_WARPS);
         }
+        for (int d = 0; d < BULK_SCHED_DEPTH; ++d) {
+            ptx::mbar_init(&sh->sched_full[d], 1);
+            ptx::mbar_init(&sh->sched_empty[d], BULK_ITEM_READERS);
+        }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&sh->io_full[b], 1);
             ptx::mbar_init(&sh->io_empty[b], 1);
@@ -458,15 +489,47 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                               : reinterpret_cast<unsigned char *>(io_tile(b, 0));
     };
 
-    TileWalk walk(p, TILE);
+    ItemWalk walk(sh, p.error_word, TILE, lane);
     long long k0;
     unsigned t = 0;  // tiles seen by this role
     RingPos q;       // ring position of this role
 
-    if (warp == BULK_COMPUTE_WARPS) {
+    if (warp == BULK_COMPUTE_WARPS + 2) {
+        // ------------------------------------------------------------------ scheduler warp
+        if (lane == 0) {
+            int slot = 0;
+            unsigned phase = 0;
+            for (;;) {
+                if (!bounded_wait(&sh->sched_empty[slot], phase ^ 1u, p.error_word, 8)) break;
+                const int item = atomicAdd(p.work_counter, 1);
+                int item_pass = -1;
+                long long b = 0, e = 0;
+                if (item < p.total_items) {
+                    // last pass whose first item is <= item (passes without items sort before it)
+                    int lo = 0, hi = p.num_passes - 1;
+                    while (lo < hi) {
+                        const int mid = (lo + hi + 1) >> 1;
+                        if (p.passes[mid].item_first <= item) lo = mid; else hi = mid - 1;
+                    }
+                    const PassDev ps = p.passes[lo];
+                    const long long first_tile = (long long)(item - ps.item_first) * ps.tiles_per_item;
+                    const long long last_tile = min(first_tile + ps.tiles_per_item, ps.bulk_tiles);
+                    item_pass = lo;
+                    b = first_tile * TILE;
+                    e = last_tile * TILE;
+                }
+                sh->sched_pass[slot] = item_pass;
+                sh->sched_begin[slot] = b;
+                sh->sched_end[slot] = e;
+                ptx::mbar_arrive(&sh->sched_full[slot]);
+                if (item_pass < 0) break;
+                if (++slot == BULK_SCHED_DEPTH) { slot = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == BULK_COMPUTE_WARPS) {
         // ------------------------------------------------------------------ load warp
         bool ok = true;
-        while (ok && walk.next(k0)) {
+        while (ok && walk.next(k0, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = t & 1;
             if (lane == 0) {
@@ -528,7 +591,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
     } else if (warp == BULK_COMPUTE_WARPS + 1) {
         // ------------------------------------------------------------------ store warp
         bool ok = true;
-        while (ok && walk.next(k0)) {
+        while (ok && walk.next(k0, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = t & 1;
             ok = bounded_wait(&sh->out_ready[b], (t >> 1) & 1, p.error_word, 4);
@@ -557,7 +620,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
         // ------------------------------------------------------------------ compute warps
         const int ct = threadIdx.x;  // 0 .. BULK_COMPUTE_THREADS-1
         bool ok = true;
-        while (ok && walk.next(k0)) {
+        while (ok && walk.next(k0, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = t & 1;
             ok = bounded_wait(&sh->io_full[b], (t >> 1) & 1, p.error_word, 5);
