@@ -51,7 +51,8 @@ enum {
     DIPACO_ENOMEM = -3,   /* host or device allocation failed                                   */
     DIPACO_ESTATE = -4,   /* call not allowed in the context's current state                    */
     DIPACO_ETIMEOUT = -5, /* a bounded wait inside a kernel ran out (reported by device_status) */
-    DIPACO_ENODEV = -6    /* the context was created without a device (plan only)               */
+    DIPACO_ENODEV = -6,   /* the context was created without a device (plan only)               */
+    DIPACO_ELIMIT = -7    /* a size exceeds a fixed limit of the entry point (static scratch)   */
 };
 
 /* kernel selection for dipaco_set_kernel */
@@ -184,6 +185,48 @@ int dipaco_plan_split(const dipaco_ctx *ctx, const uint8_t *reported, int32_t nu
                       int64_t *seg_end, int32_t *cta_first);
 
 int dipaco_destroy(dipaco_ctx *ctx);
+
+/*
+ * Synchronise ONE module without allocating anything.  (The paper has no counterpart for this
+ * entry point; it exists for the sake of its callers.)
+ *
+ * Who needs it: code that is not allowed to touch the device allocator.  Examples are a process
+ * that has handed all device memory to a pool of its own at start-up, so that a later cudaMalloc
+ * simply fails, and a latency-critical loop that cannot accept the device-wide synchronisation
+ * that cudaMalloc and cudaFree imply.  Such callers cannot use dipaco_create (it allocates
+ * tables, and in chunked mode the partial-sum scratch).  This function takes everything as
+ * arguments, passes the per-chunk tables inside the kernel arguments and keeps the partial sums
+ * in a static device array that is part of the library image.  It calls no cudaMalloc, cudaFree,
+ * cudaMallocHost or any other allocating routine, on the device or on the host heap.
+ *
+ * What it computes: the same result, bit for bit, as dipaco_outer_sync on a grid with a single
+ * level and a single module shared by num_paths paths, walked in chunks of chunk_paths.
+ *   theta, momentum   device, fp32 [numel]; in/out
+ *   numel             0 <= numel <= DIPACO_STATIC_MAX_NUMEL (4 Mi parameters = 16 MiB of partial
+ *                     sums); larger sizes are refused with DIPACO_ELIMIT and nothing is launched
+ *   num_paths         >= 1
+ *   copy_ptrs         HOST array [num_paths] of DEVICE pointers, each a copy of the module
+ *                     ([numel] of path_dtype); in/out, every copy is overwritten with cast(theta')
+ *   path_weights      HOST [num_paths] raw weights >= 0 or NULL = uniform
+ *   reported          HOST [num_paths], nonzero = reported, or NULL = all
+ *   chunk_paths       1..32 copies per chunk
+ *   device            CUDA device that owns all the buffers; made current during the call
+ *   cuda_stream       stream the kernels are launched on (asynchronous)
+ *
+ * The static array: 16 MiB per GPU, held from the moment the library's CUDA module is loaded on
+ * that GPU until the process exits, whether or not this function is ever called again.  The
+ * first call on each device looks up the array's device address (cudaGetSymbolAddress); make
+ * that first call before any stream capture begins.  All calls on one device share the array
+ * and it keeps whatever the last call left in it: each call starts its sums from zero in the
+ * kernel, so stale contents are never read, but two calls that overlap on the GPU (different
+ * streams, or different host threads) race on it and must be serialised by the caller.
+ */
+#define DIPACO_STATIC_MAX_NUMEL (4 * 1024 * 1024)
+int dipaco_module_sync_static(float *theta, float *momentum, int64_t numel, int32_t num_paths,
+                              void *const *copy_ptrs, const float *path_weights,
+                              const uint8_t *reported, float outer_lr, float outer_momentum,
+                              int32_t path_dtype, int32_t chunk_paths, int32_t device,
+                              void *cuda_stream);
 
 const char *dipaco_strerror(int status);
 

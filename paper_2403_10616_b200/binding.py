@@ -26,6 +26,8 @@ DIPACO_ENOMEM = -3
 DIPACO_ESTATE = -4
 DIPACO_ETIMEOUT = -5
 DIPACO_ENODEV = -6
+DIPACO_ELIMIT = -7
+DIPACO_STATIC_MAX_NUMEL = 4 * 1024 * 1024
 
 DIPACO_KERNEL_AUTO = 0
 DIPACO_KERNEL_VECTOR = 1
@@ -36,7 +38,7 @@ EXPORTS = [
     "dipaco_sync_begin", "dipaco_sync_accumulate", "dipaco_sync_writeback", "dipaco_sync_end",
     "dipaco_outer_sync_host", "dipaco_set_weights", "dipaco_set_kernel", "dipaco_set_tuning",
     "dipaco_device_status", "dipaco_launch_count", "dipaco_plan_module", "dipaco_plan_offsets",
-    "dipaco_plan_chunks", "dipaco_plan_split",
+    "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
 ]
 
 _lib = None
@@ -79,6 +81,7 @@ def load() -> ctypes.CDLL:
     lib.dipaco_plan_offsets.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.dipaco_plan_chunks.argtypes = [vp, vp, vp]
     lib.dipaco_plan_split.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, vp]
+    lib.dipaco_module_sync_static.argtypes = [vp, vp, i64, i32, vp, vp, vp, f32, f32, i32, i32, i32, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("dipaco_strerror", "dipaco_launch_count"):
@@ -242,6 +245,23 @@ def dipaco_plan_split(ctx, num_ctas, tile, reported=None, capacity=1 << 16):
     if n < 0:
         raise DipacoError(n, "dipaco_plan_split")
     return lvl[:n].copy(), mod[:n].copy(), beg[:n].copy(), end[:n].copy(), first
+
+
+def dipaco_module_sync_static(theta_ptr, momentum_ptr, numel, copy_ptrs, path_weights=None,
+                              reported=None, outer_lr=0.7, outer_momentum=0.9,
+                              path_dtype=DIPACO_F32, chunk_paths=8, device=0, stream=None) -> None:
+    """One module, no allocation: partial sums live in the library's static device array.
+
+    For callers that may not use the device allocator; see the declaration in dipaco.h for the
+    size limit, the shared array and the rule about the first call on a device."""
+    arr = _ptr_array(copy_ptrs)
+    w = None if path_weights is None else np.ascontiguousarray(path_weights, dtype=np.float32)
+    r = None if reported is None else np.ascontiguousarray(reported, dtype=np.uint8)
+    _check(load().dipaco_module_sync_static(theta_ptr, momentum_ptr, int(numel), len(copy_ptrs),
+                                            ctypes.cast(arr, ctypes.c_void_p), _np_ptr(w), _np_ptr(r),
+                                            float(outer_lr), float(outer_momentum), int(path_dtype),
+                                            int(chunk_paths), int(device), _stream_handle(stream)),
+           "dipaco_module_sync_static")
 
 
 # ------------------------------------------------------------------ convenience owner

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdipaco.so")
-SOURCES = ["dipaco.cu"]
-DEPENDS = ["dipaco.cu", "kernels.cuh", "plan.hpp", "host_mode.inl",
+SOURCES = ["dipaco.cu", "static_sync.cu"]
+DEPENDS = ["dipaco.cu", "static_sync.cu", "kernels.cuh", "plan.hpp", "host_mode.inl",
            os.path.join("..", "..", "include", "dipaco.h")]
 
 

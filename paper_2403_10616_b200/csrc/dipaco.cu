@@ -820,6 +820,7 @@ const char *dipaco_strerror(int status)
     case DIPACO_ESTATE: return "call not allowed in this state";
     case DIPACO_ETIMEOUT: return "a bounded wait inside a kernel ran out";
     case DIPACO_ENODEV: return "context has no device (plan only)";
+    case DIPACO_ELIMIT: return "size exceeds the fixed limit of this entry point";
     default: return "unknown status";
     }
 }
