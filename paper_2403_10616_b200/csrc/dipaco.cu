@@ -174,6 +174,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         pd.item_first = 0;
         pd.tiles_per_item = 1;
         pd.bulk_tiles = 0;
+        pd.bulk_elems = 0;
         if ((sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) && (m.partial_off < 0 || !ctx->partial))
             return DIPACO_ESTATE;
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
@@ -206,8 +207,12 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
             }
         pd.member_count = (int)members.size() - pd.member_begin;
 
+        // The vector kernel takes full tiles; the bulk-copy kernel also takes a partial last tile
+        // as long as it is a whole number of 16-byte units of path data.
         int64_t full = 0;
-        if (aligned && ctx->kernel != DIPACO_KERNEL_SCALAR) full = m.numel / tile * tile;
+        const int64_t unit = 16 / es;
+        if (aligned && ctx->kernel == DIPACO_KERNEL_VECTOR) full = m.numel / tile * tile;
+        if (aligned && ctx->kernel == DIPACO_KERNEL_AUTO) full = m.numel / unit * unit;
         bulk_begin[i] = 0; bulk_end[i] = full;
         rag_begin[i] = full; rag_end[i] = m.numel;
     }
@@ -219,7 +224,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     int64_t bulk_tiles = 0, rag_tiles = 0;
     double bulk_bytes = 0.0;
     for (size_t i = 0; i < specs.size(); ++i) {
-        bulk_tiles += (bulk_end[i] - bulk_begin[i]) / tile;
+        bulk_tiles += (bulk_end[i] - bulk_begin[i] + tile - 1) / tile;
         bulk_bytes += pass_cost_per_elem(specs[i], es) * (double)(bulk_end[i] - bulk_begin[i]);
         rag_tiles += (rag_end[i] - rag_begin[i] + RAGGED_TILE - 1) / RAGGED_TILE;
     }
@@ -232,7 +237,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         // Work items of about equal traffic, small enough that every CTA draws many of them.
         const double target = std::min(ITEM_TARGET_BYTES, bulk_bytes / ((double)bulk_ctas * 16.0));
         for (size_t i = 0; i < specs.size(); ++i) {
-            const int64_t ntiles = (bulk_end[i] - bulk_begin[i]) / tile;
+            const int64_t ntiles = (bulk_end[i] - bulk_begin[i] + tile - 1) / tile;
             const double per_tile = pass_cost_per_elem(specs[i], es) * (double)tile;
             int64_t tpi = (int64_t)std::floor(target / per_tile + 0.5);
             if (tpi < 1) tpi = 1;
@@ -240,6 +245,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
             passes[i].item_first = (int)total_items;
             passes[i].tiles_per_item = (int)tpi;
             passes[i].bulk_tiles = ntiles;
+            passes[i].bulk_elems = bulk_end[i];
             total_items += (ntiles + tpi - 1) / tpi;
         }
         if (total_items > 0x7fff0000) return DIPACO_EINVAL;

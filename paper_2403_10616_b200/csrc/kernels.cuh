@@ -30,6 +30,8 @@ struct PassDev {
     int tiles_per_item;
     int pad;
     long long bulk_tiles;
+    long long bulk_elems;  // elements covered by the bulk-copy kernel: a multiple of 16 bytes of
+                           // path data; the last tile of the pass may be partial
 };
 
 struct ContribDev {
@@ -159,7 +161,20 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
             if constexpr (VEC == 1) {
                 th[0] = theta[k];
                 acc[0] = (pass.flags & KPASS_PARTIAL_IN) ? partial[k] : 0.0f;
-                for (int j = 0; j < pass.contrib_count; ++j) {
+                // loads of four contributors in flight, summation still in ascending order
+                int j = 0;
+                for (; j + 4 <= pass.contrib_count; j += 4) {
+                    float x[4], cf[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const ContribDev c = contribs[j + u];
+                        cf[u] = c.coeff;
+                        x[u] = PathIO<PathT>::load(static_cast<const PathT *>(c.src) + k);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) acc[0] = sync_accumulate(acc[0], cf[u], th[0], x[u]);
+                }
+                for (; j < pass.contrib_count; ++j) {
                     const ContribDev c = contribs[j];
                     const float x = PathIO<PathT>::load(static_cast<const PathT *>(c.src) + k);
                     acc[0] = sync_accumulate(acc[0], c.coeff, th[0], x);
@@ -418,13 +433,18 @@ struct ItemWalk {
         : sh(shared), error_word(err), tile(tile_elems), lane(lane_id)
     {
     }
-    // Next tile of this CTA: sets pass and k0; false when the work is exhausted (ok stays true)
-    // or a wait ran out (ok = false).  Must be called by all lanes of the warp together.
-    __device__ bool next(long long &k0, bool &ok)
+    // Next tile of this CTA: sets pass, its first element k0 and its element count n (a full tile,
+    // or the partial last tile of a pass); false when the work is exhausted (ok stays true) or a
+    // wait ran out (ok = false).  Must be called by all lanes of the warp together.
+    __device__ bool next(long long &k0, unsigned &n, bool &ok)
     {
         if (pass >= 0) {
             pos += tile;
-            if (pos < end) { k0 = pos; return true; }
+            if (pos < end) {
+                k0 = pos;
+                n = (unsigned)min(tile, end - pos);
+                return true;
+            }
         }
         ok = bounded_wait(&sh->sched_full[slot], phase, error_word, 7);
         if (!ok) return false;
@@ -436,6 +456,7 @@ struct ItemWalk {
         if (item_pass < 0) return false;
         pass = item_pass; pos = b; end = e;
         k0 = pos;
+        n = (unsigned)min(tile, end - pos);
         return true;
     }
 };
@@ -491,6 +512,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
 
     ItemWalk walk(sh, p.error_word, TILE, lane);
     long long k0;
+    unsigned n;      // elements of the current tile (partial tiles: compute runs on the whole
+                     // shared-memory tile, only the first n elements are loaded and stored)
     unsigned t = 0;  // tiles seen by this role
     RingPos q;       // ring position of this role
 
@@ -516,7 +539,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                     const long long last_tile = min(first_tile + ps.tiles_per_item, ps.bulk_tiles);
                     item_pass = lo;
                     b = first_tile * TILE;
-                    e = last_tile * TILE;
+                    e = min(last_tile * TILE, ps.bulk_elems);
                 }
                 sh->sched_pass[slot] = item_pass;
                 sh->sched_begin[slot] = b;
@@ -529,24 +552,25 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
     } else if (warp == BULK_COMPUTE_WARPS) {
         // ------------------------------------------------------------------ load warp
         bool ok = true;
-        while (ok && walk.next(k0, ok)) {
+        while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = t & 1;
             if (lane == 0) {
                 ok = bounded_wait(&sh->io_empty[b], ((t >> 1) & 1) ^ 1, p.error_word, 1);
                 if (ok) {
-                    unsigned bytes = F32_TILE_BYTES;
-                    if (pass.flags & KPASS_UPDATE) bytes += F32_TILE_BYTES;
-                    if (pass.flags & KPASS_PARTIAL_IN) bytes += F32_TILE_BYTES;
+                    const unsigned f32_bytes = n * 4u;
+                    unsigned bytes = f32_bytes;
+                    if (pass.flags & KPASS_UPDATE) bytes += f32_bytes;
+                    if (pass.flags & KPASS_PARTIAL_IN) bytes += f32_bytes;
                     ptx::mbar_arrive_expect_tx(&sh->io_full[b], bytes);
-                    ptx::bulk_load(io_tile(b, 0), p.theta + pass.theta_off + k0, F32_TILE_BYTES,
+                    ptx::bulk_load(io_tile(b, 0), p.theta + pass.theta_off + k0, f32_bytes,
                                    &sh->io_full[b]);
                     if (pass.flags & KPASS_UPDATE)
-                        ptx::bulk_load(io_tile(b, 1), p.momentum + pass.theta_off + k0,
-                                       F32_TILE_BYTES, &sh->io_full[b]);
+                        ptx::bulk_load(io_tile(b, 1), p.momentum + pass.theta_off + k0, f32_bytes,
+                                       &sh->io_full[b]);
                     if (pass.flags & KPASS_PARTIAL_IN)
-                        ptx::bulk_load(io_tile(b, 2), p.partial + pass.partial_off + k0,
-                                       F32_TILE_BYTES, &sh->io_full[b]);
+                        ptx::bulk_load(io_tile(b, 2), p.partial + pass.partial_off + k0, f32_bytes,
+                                       &sh->io_full[b]);
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -564,9 +588,10 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                         ok = bounded_wait(&sh->empty[s], q.phase ^ 1u, p.error_word, 2);
                         if (!ok) break;
                         sh->slot_coeff[s] = sh->batch_coeff[u];
-                        ptx::mbar_arrive_expect_tx(&sh->full[s], STAGE_BYTES);
+                        const unsigned path_bytes = n * (unsigned)sizeof(PathT);
+                        ptx::mbar_arrive_expect_tx(&sh->full[s], path_bytes);
                         ptx::bulk_load(ring + (size_t)s * STAGE_BYTES,
-                                       static_cast<const PathT *>(sh->batch_src[u]) + k0, STAGE_BYTES,
+                                       static_cast<const PathT *>(sh->batch_src[u]) + k0, path_bytes,
                                        &sh->full[s]);
                         q.advance(stages);
                     }
@@ -591,23 +616,23 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
     } else if (warp == BULK_COMPUTE_WARPS + 1) {
         // ------------------------------------------------------------------ store warp
         bool ok = true;
-        while (ok && walk.next(k0, ok)) {
+        while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = t & 1;
             ok = bounded_wait(&sh->out_ready[b], (t >> 1) & 1, p.error_word, 4);
             if (!ok) break;
             if (lane == 0) {
                 if (pass.flags & KPASS_UPDATE) {
-                    ptx::bulk_store(p.theta + pass.theta_off + k0, io_tile(b, 0), F32_TILE_BYTES);
-                    ptx::bulk_store(p.momentum + pass.theta_off + k0, io_tile(b, 1), F32_TILE_BYTES);
+                    ptx::bulk_store(p.theta + pass.theta_off + k0, io_tile(b, 0), n * 4u);
+                    ptx::bulk_store(p.momentum + pass.theta_off + k0, io_tile(b, 1), n * 4u);
                 }
                 if (pass.flags & KPASS_PARTIAL_OUT)
-                    ptx::bulk_store(p.partial + pass.partial_off + k0, io_tile(b, 2), F32_TILE_BYTES);
+                    ptx::bulk_store(p.partial + pass.partial_off + k0, io_tile(b, 2), n * 4u);
             }
             const unsigned char *src = cast_tile(b);
             for (int j = lane; j < pass.member_count; j += 32) {
                 PathT *dst = static_cast<PathT *>(p.members[pass.member_begin + j]) + k0;
-                ptx::bulk_store(dst, src, STAGE_BYTES);
+                ptx::bulk_store(dst, src, n * (unsigned)sizeof(PathT));
             }
             ptx::bulk_commit();
             ptx::bulk_wait_read_all();
@@ -620,7 +645,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
         // ------------------------------------------------------------------ compute warps
         const int ct = threadIdx.x;  // 0 .. BULK_COMPUTE_THREADS-1
         bool ok = true;
-        while (ok && walk.next(k0, ok)) {
+        while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = t & 1;
             ok = bounded_wait(&sh->io_full[b], (t >> 1) & 1, p.error_word, 5);

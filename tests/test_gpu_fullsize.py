@@ -9,6 +9,8 @@ regenerated inputs gives bitwise the same result (order-independent integer chec
 """
 from __future__ import annotations
 
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -46,6 +48,8 @@ def run_default(problem):
 def test_full_size_sampled_parity_properties_and_reproducibility(name):
     cfg = synth.CONFIGS[name]
     need = cfg.path_params * 2 + 8 * cfg.module_params
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < need * 1.03:
         pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
@@ -109,3 +113,6 @@ def test_full_size_sampled_parity_properties_and_reproducibility(name):
     run_default(again)
     torch.cuda.synchronize()
     assert checksums(again) == first
+    del again
+    gc.collect()
+    torch.cuda.empty_cache()

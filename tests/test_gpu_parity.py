@@ -101,9 +101,10 @@ def host_state(state):
             [helpers.tensor_to_numpy(p) for p in state[2]])
 
 
-# sizes: several tiles plus a ragged tail, all levels 16-byte aligned / deliberately misaligned
-ALIGNED = {3: (3 * 2048 + 72, 2 * 2048 + 8, 5 * 2048 + 1000),
-           5: (3 * 2048 + 72, 2 * 2048 + 8, 2048 + 1000, 4096, 4096 + 16)}
+# sizes: several tiles plus a ragged tail (the last level's tail is not a whole 16-byte unit),
+# all levels 16-byte aligned / deliberately misaligned
+ALIGNED = {3: (3 * 2048 + 72, 2 * 2048 + 8, 5 * 2048 + 1003),
+           5: (3 * 2048 + 72, 2 * 2048 + 8, 2048 + 1000, 4096, 4096 + 21)}
 ODD = {3: (50003, 50003, 50003), 5: (20003, 10001, 10001, 10001, 10001)}
 
 
