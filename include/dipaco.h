@@ -119,10 +119,14 @@ int dipaco_sync_end(dipaco_ctx *ctx);
 
 /*
  * The same synchronisation for state that lives in HOST memory (checkpoints that do not fit
- * on the device): theta, momentum [module params] and the P path copies are host buffers
- * (pinned memory gives full copy speed).  Path copies are streamed through the device in
- * chunks of chunk_paths (> 0 required) with copies overlapping the kernels; theta' and m' are
- * copied back and every path copy is overwritten with its modules' cast(theta').
+ * on the device; Section 3.3: the executor loads checkpoints and averages them as they come):
+ * theta, momentum [module params] and the P path copies are host buffers (pinned memory gives
+ * full copy speed).  The work is streamed through the device slab by slab: an element range of
+ * one module together with that range of every reporting copy is uploaded, reduced, updated and
+ * cast in one fused pass, and the result is copied back into theta, momentum and the slot of
+ * every path of the module while the next slab is already being uploaded.  Device staging is
+ * bounded by the size of chunk_paths path copies (> 0 required) plus theta and momentum.  Paths
+ * that did not report are not uploaded.  Results are bitwise those of dipaco_outer_sync.
  * Synchronous: returns when all host buffers hold the result.
  */
 int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
@@ -143,6 +147,13 @@ int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
  */
 int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
                       int32_t units_per_thread);
+
+/*
+ * Tuning of dipaco_outer_sync_host: the most bytes of path data one streamed unit uploads
+ * (0 = no cap other than the staging buffers).  Smaller units fill and drain the pipeline
+ * faster, larger ones mean fewer and larger copies.
+ */
+int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes);
 
 /*
  * Synchronise the context's last stream and report what the kernels recorded: DIPACO_OK, or
@@ -171,6 +182,15 @@ int dipaco_plan_offsets(const dipaco_ctx *ctx, int32_t level, int32_t module,
                         int64_t *theta_offset, int64_t *path_offset, int64_t *numel);
 /* Number of chunks (1 when chunk_paths = 0) and fp32 elements of partial-sum scratch. */
 int dipaco_plan_chunks(const dipaco_ctx *ctx, int32_t *num_chunks, int64_t *scratch_elems);
+
+/*
+ * Bytes that one dipaco_outer_sync on this context moves through device memory by
+ * construction (every read and write of theta, momentum, partial sums and path copies, summed
+ * over its launches), and the number of launches (tail launches not counted).  For a resident
+ * context this is the algorithmic minimum; for a chunked one it includes the partial-sum traffic.
+ */
+int dipaco_plan_traffic(const dipaco_ctx *ctx, const uint8_t *reported, int64_t *bytes,
+                        int32_t *launches);
 
 /*
  * The split of the resident-mode launch over num_ctas persistent CTAs in tiles of `tile`

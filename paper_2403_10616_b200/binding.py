@@ -39,6 +39,7 @@ EXPORTS = [
     "dipaco_outer_sync_host", "dipaco_set_weights", "dipaco_set_kernel", "dipaco_set_tuning",
     "dipaco_device_status", "dipaco_launch_count", "dipaco_plan_module", "dipaco_plan_offsets",
     "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
+    "dipaco_set_host_unit_bytes", "dipaco_plan_traffic",
 ]
 
 _lib = None
@@ -75,11 +76,13 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32]
     lib.dipaco_device_status.argtypes = [vp]
+    lib.dipaco_set_host_unit_bytes.argtypes = [vp, i64]
     lib.dipaco_launch_count.argtypes = [vp]
     lib.dipaco_launch_count.restype = i64
     lib.dipaco_plan_module.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.dipaco_plan_offsets.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.dipaco_plan_chunks.argtypes = [vp, vp, vp]
+    lib.dipaco_plan_traffic.argtypes = [vp, vp, vp, vp]
     lib.dipaco_plan_split.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp, vp, vp]
     lib.dipaco_module_sync_static.argtypes = [vp, vp, i64, i32, vp, vp, vp, f32, f32, i32, i32, i32, vp]
     for name in EXPORTS:
@@ -196,6 +199,10 @@ def dipaco_set_tuning(ctx, ctas_per_sm=0, stages=0, units_per_thread=0) -> None:
            "dipaco_set_tuning")
 
 
+def dipaco_set_host_unit_bytes(ctx, nbytes: int) -> None:
+    _check(load().dipaco_set_host_unit_bytes(ctx, int(nbytes)), "dipaco_set_host_unit_bytes")
+
+
 def dipaco_device_status(ctx) -> int:
     return int(load().dipaco_device_status(ctx))
 
@@ -229,6 +236,15 @@ def dipaco_plan_chunks(ctx):
     n, s = ctypes.c_int32(), ctypes.c_int64()
     _check(load().dipaco_plan_chunks(ctx, ctypes.addressof(n), ctypes.addressof(s)), "dipaco_plan_chunks")
     return n.value, s.value
+
+
+def dipaco_plan_traffic(ctx, reported=None):
+    """(bytes moved by one dipaco_outer_sync by construction, number of launches)."""
+    r = None if reported is None else np.ascontiguousarray(reported, dtype=np.uint8)
+    nbytes, launches = ctypes.c_int64(), ctypes.c_int32()
+    _check(load().dipaco_plan_traffic(ctx, _np_ptr(r), ctypes.addressof(nbytes),
+                                      ctypes.addressof(launches)), "dipaco_plan_traffic")
+    return nbytes.value, launches.value
 
 
 def dipaco_plan_split(ctx, num_ctas, tile, reported=None, capacity=1 << 16):

@@ -56,6 +56,7 @@ struct dipaco_ctx {
     int kernel = DIPACO_KERNEL_AUTO;
     int ctas_per_sm = 1, stages = 10, units = 2;  // bulk-copy kernel tuning (measured on B200)
     int64_t launches = 0;
+    int64_t host_unit_bytes = (int64_t)1 << 40;  // upload size cap of one unit in host mode
 
     void *dev_tables = nullptr;
     size_t dev_tables_capacity = 0;
@@ -174,7 +175,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         pd.item_first = 0;
         pd.tiles_per_item = 1;
         pd.bulk_tiles = 0;
-        pd.bulk_elems = 0;
+        pd.bulk_begin = 0;
+        pd.bulk_end = 0;
         if ((sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) && (m.partial_off < 0 || !ctx->partial))
             return DIPACO_ESTATE;
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
@@ -209,12 +211,17 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
 
         // The vector kernel takes full tiles; the bulk-copy kernel also takes a partial last tile
         // as long as it is a whole number of 16-byte units of path data.
-        int64_t full = 0;
+        const int64_t lo = sp.begin, hi = sp.end < 0 ? m.numel : sp.end;
+        if (lo < 0 || hi > m.numel || lo > hi) return DIPACO_EINVAL;
+        // a range that does not start on a 16-byte unit of both theta and the path data is
+        // handled like a misaligned module
         const int64_t unit = 16 / es;
-        if (aligned && ctx->kernel == DIPACO_KERNEL_VECTOR) full = m.numel / tile * tile;
-        if (aligned && ctx->kernel == DIPACO_KERNEL_AUTO) full = m.numel / unit * unit;
-        bulk_begin[i] = 0; bulk_end[i] = full;
-        rag_begin[i] = full; rag_end[i] = m.numel;
+        if (lo % unit != 0) aligned = false;
+        int64_t full = 0;
+        if (aligned && ctx->kernel == DIPACO_KERNEL_VECTOR) full = (hi - lo) / tile * tile;
+        if (aligned && ctx->kernel == DIPACO_KERNEL_AUTO) full = (hi - lo) / unit * unit;
+        bulk_begin[i] = lo; bulk_end[i] = lo + full;
+        rag_begin[i] = lo + full; rag_end[i] = hi;
     }
 
     std::vector<Segment> bulk_segs, rag_segs;
@@ -245,7 +252,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
             passes[i].item_first = (int)total_items;
             passes[i].tiles_per_item = (int)tpi;
             passes[i].bulk_tiles = ntiles;
-            passes[i].bulk_elems = bulk_end[i];
+            passes[i].bulk_begin = bulk_begin[i];
+            passes[i].bulk_end = bulk_end[i];
             total_items += (ntiles + tpi - 1) / tpi;
         }
         if (total_items > 0x7fff0000) return DIPACO_EINVAL;
@@ -578,6 +586,14 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
     return DIPACO_OK;
 }
 
+int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes)
+{
+    if (!ctx || bytes < 0) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ctx->host_unit_bytes = bytes == 0 ? (int64_t)1 << 40 : bytes;
+    return DIPACO_OK;
+}
+
 int dipaco_sync_begin(dipaco_ctx *ctx, float *theta, float *momentum, const uint8_t *reported,
                       void *cuda_stream)
 {
@@ -780,6 +796,38 @@ int dipaco_plan_chunks(const dipaco_ctx *ctx, int32_t *num_chunks, int64_t *scra
     if (!ctx) return DIPACO_EINVAL;
     if (num_chunks) *num_chunks = ctx->grid.num_chunks;
     if (scratch_elems) *scratch_elems = ctx->grid.scratch_elems;
+    return DIPACO_OK;
+}
+
+int dipaco_plan_traffic(const dipaco_ctx *ctx, const uint8_t *reported, int64_t *bytes,
+                        int32_t *launches)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    try {
+        const Grid &g = ctx->grid;
+        std::vector<ModuleCoeffs> mc(g.modules.size());
+        for (size_t id = 0; id < mc.size(); ++id) module_coeffs(g, g.modules[id], reported, mc[id]);
+        double total = 0.0;
+        int count = 0;
+        std::vector<PassSpec> specs;
+        auto add = [&]() {
+            if (specs.empty()) return;
+            ++count;
+            for (const PassSpec &sp : specs)
+                total += pass_cost_per_elem(sp, ctx->elem_size) * (double)g.modules[sp.module].numel;
+        };
+        if (g.num_chunks <= 1) {
+            plan_resident(g, mc, specs);
+            add();
+        } else {
+            for (int c = 0; c < g.num_chunks; ++c) { plan_accumulate(g, mc, c, specs); add(); }
+            for (int c = 0; c < g.num_chunks; ++c) { plan_writeback(g, mc, c, true, specs); add(); }
+        }
+        if (bytes) *bytes = (int64_t)total;
+        if (launches) *launches = count;
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
     return DIPACO_OK;
 }
 

@@ -1,45 +1,51 @@
 // dipaco_outer_sync_host: the synchronisation for state kept in host memory.
 // Included by dipaco.cu (inside its translation unit, after the launch helpers).
 //
-// Reporting path copies are streamed host -> device in chunks of chunk_paths through two device
-// buffers (the copy of chunk c+1 overlaps the kernel of chunk c).  The chunk kernels only read
-// the copies; as soon as a module's last reporting path has been accumulated the module is
-// updated, its value is cast once into a device array shaped like theta (bf16 paths only) and
-// copied device -> host into the slot of every path through the module, while later chunks are
-// still being uploaded.  Paths that did not report are never uploaded.
+// Slab-ordered streaming.  The work is cut into units: an element range [a, b) of one module
+// together with that range of EVERY reporting copy of the module.  A unit is therefore complete
+// in itself: one fused pass (reduce in ascending path id + Nesterov + cast) finishes it, no
+// partial sums are carried, and its result can leave the device at once.  Per unit:
+//     H2D  theta[a:b], m[a:b] and the [a:b) piece of each reporting copy  -> staging buffer
+//     kernel  the resident-mode pass on [a, b), reading the staged pieces, writing theta', m'
+//             in place and cast(theta') into a small output buffer
+//     D2H  theta'[a:b], m'[a:b], and the output buffer into the slot of every path of the module
+// Units are double-buffered over three streams, so the upload of unit n+1, the kernel of unit n
+// and the download of unit n-1 overlap; a step costs about max(H2D bytes, D2H bytes) / PCIe rate.
+// The staging memory is bounded by chunk_paths path copies.  Paths that did not report are never
+// uploaded.  Bitwise identical to the resident mode: same pass, same order.
 
 namespace {
 
 struct HostMode {
-    float *theta_d = nullptr, *momentum_d = nullptr;
-    void *chunk_buf[2] = {nullptr, nullptr};
-    void *cast_d = nullptr;  // module values in the path dtype (bf16 paths only)
-    cudaStream_t copy_stream = nullptr, d2h_stream = nullptr;
-    cudaEvent_t h2d_done[2] = {nullptr, nullptr};
-    cudaEvent_t buf_free[2] = {nullptr, nullptr};
+    float *theta_d = nullptr, *momentum_d = nullptr;  // full module state on the device
+    char *stage_in[2] = {nullptr, nullptr};           // staged pieces of path copies
+    char *stage_out[2] = {nullptr, nullptr};          // cast(theta') of the unit (bf16 paths)
+    size_t stage_in_bytes = 0, stage_out_bytes = 0;
+    cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    cudaEvent_t in_ready[2] = {nullptr, nullptr};    // upload of the unit in this buffer finished
+    cudaEvent_t kernel_done[2] = {nullptr, nullptr}; // kernel finished: input reusable, output ready
+    cudaEvent_t out_done[2] = {nullptr, nullptr};    // download finished: output buffer reusable
     cudaEvent_t main_ready = nullptr;
-    std::vector<cudaEvent_t> finalised;  // one per chunk + one for the modules nobody reported to
 };
 
 void host_mode_release(dipaco_ctx *ctx)
 {
     HostMode *h = ctx->host_mode;
     if (!h) return;
-    if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
-    if (h->d2h_stream) cudaStreamSynchronize(h->d2h_stream);
+    if (h->in_stream) cudaStreamSynchronize(h->in_stream);
+    if (h->out_stream) cudaStreamSynchronize(h->out_stream);
     if (h->theta_d) cudaFree(h->theta_d);
     if (h->momentum_d) cudaFree(h->momentum_d);
     for (int b = 0; b < 2; ++b) {
-        if (h->chunk_buf[b]) cudaFree(h->chunk_buf[b]);
-        if (h->h2d_done[b]) cudaEventDestroy(h->h2d_done[b]);
-        if (h->buf_free[b]) cudaEventDestroy(h->buf_free[b]);
+        if (h->stage_in[b]) cudaFree(h->stage_in[b]);
+        if (h->stage_out[b]) cudaFree(h->stage_out[b]);
+        if (h->in_ready[b]) cudaEventDestroy(h->in_ready[b]);
+        if (h->kernel_done[b]) cudaEventDestroy(h->kernel_done[b]);
+        if (h->out_done[b]) cudaEventDestroy(h->out_done[b]);
     }
-    if (h->cast_d) cudaFree(h->cast_d);
     if (h->main_ready) cudaEventDestroy(h->main_ready);
-    for (cudaEvent_t e : h->finalised)
-        if (e) cudaEventDestroy(e);
-    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
-    if (h->d2h_stream) cudaStreamDestroy(h->d2h_stream);
+    if (h->in_stream) cudaStreamDestroy(h->in_stream);
+    if (h->out_stream) cudaStreamDestroy(h->out_stream);
     delete h;
     ctx->host_mode = nullptr;
 }
@@ -51,81 +57,43 @@ int host_mode_prepare(dipaco_ctx *ctx)
     HostMode *h = new (std::nothrow) HostMode();
     if (!h) return DIPACO_ENOMEM;
     ctx->host_mode = h;
+    const int es = ctx->elem_size;
     const size_t module_bytes = std::max<size_t>((size_t)g.module_params * sizeof(float), 16);
-    const size_t path_bytes = align_up((size_t)g.params_per_path * ctx->elem_size, 256);
-    const size_t chunk_bytes = std::max<size_t>(path_bytes * (size_t)g.chunk_paths, 16);
+    // two input buffers that together hold chunk_paths path copies
+    const size_t tile_bytes = (size_t)tile_elems(ctx) * es;
+    size_t in_bytes = (size_t)g.chunk_paths * (size_t)g.params_per_path * es / 2;
+    size_t max_contrib = 1;
+    int64_t max_numel = 1;
+    for (const ModuleGeom &m : g.modules) {
+        max_contrib = std::max(max_contrib, m.members.size());
+        max_numel = std::max(max_numel, m.numel);
+    }
+    in_bytes = std::max(in_bytes, max_contrib * tile_bytes);  // at least one tile of every copy
+    h->stage_in_bytes = align_up(in_bytes, 256);
+    // the largest unit is bounded by a whole module and by stage_in_bytes / (1 copy)
+    const size_t out_elems = std::min<size_t>((size_t)max_numel, h->stage_in_bytes / es);
+    h->stage_out_bytes = align_up(std::max<size_t>(out_elems * es, 256), 256);
     bool ok = cudaMalloc(&h->theta_d, module_bytes) == cudaSuccess &&
-              cudaMalloc(&h->momentum_d, module_bytes) == cudaSuccess &&
-              cudaMalloc(&h->chunk_buf[0], chunk_bytes) == cudaSuccess &&
-              cudaMalloc(&h->chunk_buf[1], chunk_bytes) == cudaSuccess;
-    if (ok && ctx->elem_size != 4)
-        ok = cudaMalloc(&h->cast_d, std::max<size_t>((size_t)g.module_params * ctx->elem_size, 16)) ==
-             cudaSuccess;
+              cudaMalloc(&h->momentum_d, module_bytes) == cudaSuccess;
+    for (int b = 0; ok && b < 2; ++b) {
+        ok = cudaMalloc(&h->stage_in[b], h->stage_in_bytes) == cudaSuccess;
+        if (ok && es != 4) ok = cudaMalloc(&h->stage_out[b], h->stage_out_bytes) == cudaSuccess;
+    }
     if (!ok) {
         cudaGetLastError();
         host_mode_release(ctx);
         return DIPACO_ENOMEM;
     }
-    ok = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
-         cudaStreamCreateWithFlags(&h->d2h_stream, cudaStreamNonBlocking) == cudaSuccess &&
+    ok = cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking) == cudaSuccess &&
+         cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking) == cudaSuccess &&
          cudaEventCreateWithFlags(&h->main_ready, cudaEventDisableTiming) == cudaSuccess;
     for (int b = 0; ok && b < 2; ++b)
-        ok = cudaEventCreateWithFlags(&h->h2d_done[b], cudaEventDisableTiming) == cudaSuccess &&
-             cudaEventCreateWithFlags(&h->buf_free[b], cudaEventDisableTiming) == cudaSuccess;
-    h->finalised.assign((size_t)g.num_chunks + 1, nullptr);
-    for (size_t i = 0; ok && i < h->finalised.size(); ++i)
-        ok = cudaEventCreateWithFlags(&h->finalised[i], cudaEventDisableTiming) == cudaSuccess;
+        ok = cudaEventCreateWithFlags(&h->in_ready[b], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&h->kernel_done[b], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&h->out_done[b], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
         host_mode_release(ctx);
         return DIPACO_ECUDA;
-    }
-    return DIPACO_OK;
-}
-
-// Cast the given modules' current theta into cast_d (bf16 paths) on `stream`, then copy the new
-// value of each module to the host: theta', m' (if updated) and the slot of every member path.
-int host_mode_emit(dipaco_ctx *ctx, const std::vector<int> &module_ids, bool updated,
-                   float *theta_host, float *momentum_host, void *const *path_ptrs_host,
-                   cudaStream_t stream, cudaEvent_t done_event)
-{
-    HostMode *h = ctx->host_mode;
-    const Grid &g = ctx->grid;
-    const int es = ctx->elem_size;
-    if (module_ids.empty()) return DIPACO_OK;
-    if (h->cast_d) {
-        std::vector<LaunchRequest> reqs(1);
-        for (int id : module_ids) {
-            PassSpec sp;
-            sp.module = id;
-            sp.flags = 0;
-            reqs[0].specs.push_back(sp);
-            reqs[0].extra_dst.push_back(
-                {static_cast<char *>(h->cast_d) + (size_t)g.modules[id].theta_off * es});
-        }
-        reqs[0].lookup = PtrLookup{nullptr, 0, 0};
-        const int rc = run_launches(ctx, reqs, h->theta_d, h->momentum_d, stream);
-        if (rc != DIPACO_OK) return rc;
-    }
-    if (cudaEventRecord(done_event, stream) != cudaSuccess) return DIPACO_ECUDA;
-    if (cudaStreamWaitEvent(h->d2h_stream, done_event, 0) != cudaSuccess) return DIPACO_ECUDA;
-    for (int id : module_ids) {
-        const ModuleGeom &m = g.modules[id];
-        const size_t fbytes = (size_t)m.numel * sizeof(float);
-        if (updated) {
-            if (cudaMemcpyAsync(theta_host + m.theta_off, h->theta_d + m.theta_off, fbytes,
-                                cudaMemcpyDeviceToHost, h->d2h_stream) != cudaSuccess ||
-                cudaMemcpyAsync(momentum_host + m.theta_off, h->momentum_d + m.theta_off, fbytes,
-                                cudaMemcpyDeviceToHost, h->d2h_stream) != cudaSuccess)
-                return DIPACO_ECUDA;
-        }
-        const char *src = h->cast_d ? static_cast<const char *>(h->cast_d) + (size_t)m.theta_off * es
-                                    : reinterpret_cast<const char *>(h->theta_d + m.theta_off);
-        for (int i : m.members) {
-            char *dst = static_cast<char *>(path_ptrs_host[i]) + (size_t)m.path_off * es;
-            if (cudaMemcpyAsync(dst, src, (size_t)m.numel * es, cudaMemcpyDeviceToHost,
-                                h->d2h_stream) != cudaSuccess)
-                return DIPACO_ECUDA;
-        }
     }
     return DIPACO_OK;
 }
@@ -138,69 +106,112 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
     HostMode *h = ctx->host_mode;
     const Grid &g = ctx->grid;
     const int es = ctx->elem_size;
-    const size_t module_bytes = (size_t)g.module_params * sizeof(float);
-    const size_t path_bytes = (size_t)g.params_per_path * es;
-    const size_t path_stride = align_up(path_bytes, 256);
+    const int64_t tile = tile_elems(ctx);
     compute_all_coeffs(ctx, reported);
 
-    if (module_bytes > 0 &&
-        (cudaMemcpyAsync(h->theta_d, theta_host, module_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-         cudaMemcpyAsync(h->momentum_d, momentum_host, module_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess))
-        return DIPACO_ECUDA;
     // the side streams must not run ahead of work queued earlier on the caller's stream
     if (cudaEventRecord(h->main_ready, stream) != cudaSuccess ||
-        cudaStreamWaitEvent(h->copy_stream, h->main_ready, 0) != cudaSuccess ||
-        cudaStreamWaitEvent(h->d2h_stream, h->main_ready, 0) != cudaSuccess)
+        cudaStreamWaitEvent(h->in_stream, h->main_ready, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(h->out_stream, h->main_ready, 0) != cudaSuccess)
         return DIPACO_ECUDA;
 
-    std::vector<void *> chunk_ptrs((size_t)g.chunk_paths);
-    for (int c = 0; c < g.num_chunks; ++c) {
-        const int b = c & 1;
-        const int first = chunk_first(g, c), n = chunk_count(g, c);
-        if (c >= 2 && cudaStreamWaitEvent(h->copy_stream, h->buf_free[b], 0) != cudaSuccess)
-            return DIPACO_ECUDA;
-        for (int j = 0; j < n; ++j) {
-            chunk_ptrs[(size_t)j] = static_cast<char *>(h->chunk_buf[b]) + (size_t)j * path_stride;
-            const int i = first + j;
-            if (reported && !reported[i]) continue;
-            if (path_bytes > 0 &&
-                cudaMemcpyAsync(chunk_ptrs[(size_t)j], path_ptrs_host[i], path_bytes,
-                                cudaMemcpyHostToDevice, h->copy_stream) != cudaSuccess)
+    std::vector<void *> by_path((size_t)g.P, nullptr);
+    long long unit_index = 0;
+    for (size_t id = 0; id < g.modules.size(); ++id) {
+        const ModuleGeom &m = g.modules[id];
+        const ModuleCoeffs &mc = ctx->coeffs[id];
+        if (m.members.empty() || m.numel == 0) continue;
+        const size_t ncon = mc.contributors.size();
+        // elements per unit: every reporting copy's piece must fit the input buffer
+        // and a unit uploads at most HOST_UNIT_BYTES so that the pipeline fills and drains quickly
+        const size_t in_budget = std::max<size_t>(std::min(h->stage_in_bytes, (size_t)ctx->host_unit_bytes),
+                                                  ncon * (size_t)tile * es);
+        int64_t slab = m.numel;
+        if (ncon > 0 && ncon * align_up((size_t)m.numel * es, 256) > in_budget) {
+            const int64_t fit = (int64_t)(in_budget / (ncon * (size_t)es));
+            slab = fit / tile * tile;  // a tile's bytes are a multiple of the 256-byte piece stride
+        }
+        if ((size_t)slab * es > h->stage_out_bytes)
+            slab = (int64_t)(h->stage_out_bytes / (size_t)es) / tile * tile;
+        if (slab < 1) return DIPACO_ENOMEM;
+        for (int64_t a = 0; a < m.numel; a += slab, ++unit_index) {
+            const int64_t b = std::min<int64_t>(m.numel, a + slab);
+            const int buf = (int)(unit_index & 1);
+            const size_t piece = (size_t)(b - a) * es;
+            const size_t piece_stride = align_up(piece, 256);
+            const size_t fbytes = (size_t)(b - a) * sizeof(float);
+
+            // ---- upload (in_stream): wait until the kernel of unit n-2 released this buffer
+            if (unit_index >= 2 && cudaStreamWaitEvent(h->in_stream, h->kernel_done[buf], 0) != cudaSuccess)
                 return DIPACO_ECUDA;
-        }
-        if (cudaEventRecord(h->h2d_done[b], h->copy_stream) != cudaSuccess ||
-            cudaStreamWaitEvent(stream, h->h2d_done[b], 0) != cudaSuccess)
-            return DIPACO_ECUDA;
+            if (cudaMemcpyAsync(h->theta_d + m.theta_off + a, theta_host + m.theta_off + a, fbytes,
+                                cudaMemcpyHostToDevice, h->in_stream) != cudaSuccess)
+                return DIPACO_ECUDA;
+            if (mc.update &&
+                cudaMemcpyAsync(h->momentum_d + m.theta_off + a, momentum_host + m.theta_off + a, fbytes,
+                                cudaMemcpyHostToDevice, h->in_stream) != cudaSuccess)
+                return DIPACO_ECUDA;
+            for (size_t j = 0; j < ncon; ++j) {
+                const int i = mc.contributors[j];
+                char *dst = h->stage_in[buf] + j * piece_stride;
+                const char *src = static_cast<const char *>(path_ptrs_host[i]) + (size_t)(m.path_off + a) * es;
+                if (cudaMemcpyAsync(dst, src, piece, cudaMemcpyHostToDevice, h->in_stream) != cudaSuccess)
+                    return DIPACO_ECUDA;
+                // virtual base: base + (path_off + k) * es lands on the staged piece for k in [a, b)
+                by_path[(size_t)i] = reinterpret_cast<void *>(reinterpret_cast<uintptr_t>(dst) -
+                                                              (uintptr_t)(m.path_off + a) * es);
+            }
+            if (cudaEventRecord(h->in_ready[buf], h->in_stream) != cudaSuccess ||
+                cudaStreamWaitEvent(stream, h->in_ready[buf], 0) != cudaSuccess)
+                return DIPACO_ECUDA;
 
-        std::vector<LaunchRequest> reqs(1);
-        plan_accumulate(g, ctx->coeffs, c, reqs[0].specs);
-        std::vector<int> done_here;
-        for (PassSpec &sp : reqs[0].specs) {
-            sp.members.clear();  // results leave through the cast array, not the chunk buffers
-            if (sp.flags & PASS_UPDATE) done_here.push_back(sp.module);
+            // ---- kernel (caller's stream): the output buffer must have been downloaded
+            if (unit_index >= 2 && cudaStreamWaitEvent(stream, h->out_done[buf], 0) != cudaSuccess)
+                return DIPACO_ECUDA;
+            const bool need_kernel = mc.update || es != 4;
+            if (need_kernel) {
+                std::vector<LaunchRequest> reqs(1);
+                PassSpec sp;
+                sp.module = (int)id;
+                sp.flags = mc.update ? PASS_UPDATE : 0;
+                sp.contributors = mc.contributors;
+                sp.coeff = mc.coeff;
+                sp.begin = a;
+                sp.end = b;
+                reqs[0].specs.push_back(std::move(sp));
+                if (es != 4)
+                    reqs[0].extra_dst.push_back({reinterpret_cast<void *>(
+                        reinterpret_cast<uintptr_t>(h->stage_out[buf]) - (uintptr_t)a * es)});
+                reqs[0].lookup = PtrLookup{by_path.data(), 0, g.P};
+                rc = run_launches(ctx, reqs, h->theta_d, h->momentum_d, stream);
+                if (rc != DIPACO_OK) return rc;
+            }
+            for (size_t j = 0; j < ncon; ++j) by_path[(size_t)mc.contributors[j]] = nullptr;
+            if (cudaEventRecord(h->kernel_done[buf], stream) != cudaSuccess ||
+                cudaStreamWaitEvent(h->out_stream, h->kernel_done[buf], 0) != cudaSuccess)
+                return DIPACO_ECUDA;
+
+            // ---- download (out_stream)
+            if (mc.update) {
+                if (cudaMemcpyAsync(theta_host + m.theta_off + a, h->theta_d + m.theta_off + a, fbytes,
+                                    cudaMemcpyDeviceToHost, h->out_stream) != cudaSuccess ||
+                    cudaMemcpyAsync(momentum_host + m.theta_off + a, h->momentum_d + m.theta_off + a,
+                                    fbytes, cudaMemcpyDeviceToHost, h->out_stream) != cudaSuccess)
+                    return DIPACO_ECUDA;
+            }
+            const char *out_src = es != 4 ? h->stage_out[buf]
+                                          : reinterpret_cast<const char *>(h->theta_d + m.theta_off + a);
+            for (int i : m.members) {
+                char *dst = static_cast<char *>(path_ptrs_host[i]) + (size_t)(m.path_off + a) * es;
+                if (cudaMemcpyAsync(dst, out_src, piece, cudaMemcpyDeviceToHost, h->out_stream) != cudaSuccess)
+                    return DIPACO_ECUDA;
+            }
+            if (cudaEventRecord(h->out_done[buf], h->out_stream) != cudaSuccess) return DIPACO_ECUDA;
         }
-        reqs[0].lookup = PtrLookup{chunk_ptrs.data(), first, n};
-        if (!reqs[0].specs.empty()) {
-            rc = run_launches(ctx, reqs, h->theta_d, h->momentum_d, stream);
-            if (rc != DIPACO_OK) return rc;
-        }
-        if (cudaEventRecord(h->buf_free[b], stream) != cudaSuccess) return DIPACO_ECUDA;
-        rc = host_mode_emit(ctx, done_here, true, theta_host, momentum_host, path_ptrs_host, stream,
-                            h->finalised[(size_t)c]);
-        if (rc != DIPACO_OK) return rc;
     }
-    // modules nobody reported to: theta and m stay, their copies are reset to cast(theta)
-    std::vector<int> untouched;
-    for (size_t id = 0; id < g.modules.size(); ++id)
-        if (!ctx->coeffs[id].update && !g.modules[id].members.empty() && g.modules[id].numel > 0)
-            untouched.push_back((int)id);
-    rc = host_mode_emit(ctx, untouched, false, theta_host, momentum_host, path_ptrs_host, stream,
-                        h->finalised[(size_t)g.num_chunks]);
-    if (rc != DIPACO_OK) return rc;
-
-    if (cudaStreamSynchronize(h->copy_stream) != cudaSuccess ||
+    if (cudaStreamSynchronize(h->in_stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess ||
-        cudaStreamSynchronize(h->d2h_stream) != cudaSuccess)
+        cudaStreamSynchronize(h->out_stream) != cudaSuccess)
         return DIPACO_ECUDA;
     return DIPACO_OK;
 }

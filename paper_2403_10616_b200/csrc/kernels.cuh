@@ -30,8 +30,9 @@ struct PassDev {
     int tiles_per_item;
     int pad;
     long long bulk_tiles;
-    long long bulk_elems;  // elements covered by the bulk-copy kernel: a multiple of 16 bytes of
-                           // path data; the last tile of the pass may be partial
+    long long bulk_begin;  // element range [bulk_begin, bulk_end) of the module that the bulk-copy
+    long long bulk_end;    // kernel covers: whole 16-byte units of path data; the last tile of the
+                           // pass may be partial
 };
 
 struct ContribDev {
@@ -538,8 +539,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                     const long long first_tile = (long long)(item - ps.item_first) * ps.tiles_per_item;
                     const long long last_tile = min(first_tile + ps.tiles_per_item, ps.bulk_tiles);
                     item_pass = lo;
-                    b = first_tile * TILE;
-                    e = min(last_tile * TILE, ps.bulk_elems);
+                    b = ps.bulk_begin + first_tile * TILE;
+                    e = min(ps.bulk_begin + last_tile * TILE, ps.bulk_end);
                 }
                 sh->sched_pass[slot] = item_pass;
                 sh->sched_begin[slot] = b;

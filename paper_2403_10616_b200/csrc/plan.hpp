@@ -137,6 +137,7 @@ struct PassSpec {
     std::vector<int> contributors; // path ids read in this launch
     std::vector<float> coeff;
     std::vector<int> members;      // path ids written in this launch
+    int64_t begin = 0, end = -1;   // element range of the module ([0, numel) when end < 0)
 };
 
 // Resident mode: one launch covers every module completely.

@@ -39,7 +39,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_strerror_names_every_status():
-    for code in (0, -1, -2, -3, -4, -5, -6):
+    for code in (0, -1, -2, -3, -4, -5, -6, -7):
         assert B.strerror(code) != "unknown status"
     assert B.strerror(-99) == "unknown status"
 
@@ -213,4 +213,20 @@ def test_split_covers_every_full_tile_once_and_balances_cost(name, numel, ctas):
             cost[b] += per_level[lvl[i]] * (end[i] - beg[i])
     heaviest_tile = max(per_level) * tile
     assert cost.max() - cost.sum() / ctas <= 1.01 * heaviest_tile
+    B.dipaco_destroy(ctx)
+
+
+def test_planned_traffic_of_resident_mode_is_the_algorithmic_minimum():
+    for name in ("grid16x16", "grid16x16-masked", "grid4x4x4x4", "grid4x4"):
+        cfg = synth.CONFIGS[name]
+        r = synth.reported_mask(cfg)
+        ctx = plan_ctx(cfg, weights=synth.path_weights(cfg))
+        nbytes, launches = B.dipaco_plan_traffic(ctx, r)
+        assert launches == 1 and nbytes == synth.algorithmic_bytes(cfg, r)
+        B.dipaco_destroy(ctx)
+    # walking the 16x16 workload in chunks of 32 paths carries partial sums: ~1.5x the traffic
+    cfg = synth.CONFIGS["grid16x16"]
+    ctx = plan_ctx(cfg, chunk_paths=32)
+    nbytes, launches = B.dipaco_plan_traffic(ctx)
+    assert launches == 15 and 1.4 < nbytes / synth.algorithmic_bytes(cfg) < 1.6
     B.dipaco_destroy(ctx)
