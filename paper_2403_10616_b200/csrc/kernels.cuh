@@ -60,7 +60,8 @@ struct LaunchParams {
     // bulk-copy kernel only
     int num_passes;
     int total_items;
-    int *work_counter;  // zeroed before the launch; CTAs draw work items from it
+    int *work_counter;  // [0]: next work item, [1]: CTAs that finished drawing; both zero before the
+                        // launch, and reset to zero by the last CTA so the next launch can reuse them
 };
 
 // ------------------------------------------------------------------------------------------
@@ -546,7 +547,14 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                 sh->sched_begin[slot] = b;
                 sh->sched_end[slot] = e;
                 ptx::mbar_arrive(&sh->sched_full[slot]);
-                if (item_pass < 0) break;
+                if (item_pass < 0) {
+                    // nobody draws after its own sentinel: the last CTA here re-arms the counters
+                    if (atomicAdd(p.work_counter + 1, 1) == (int)gridDim.x - 1) {
+                        p.work_counter[0] = 0;
+                        p.work_counter[1] = 0;
+                    }
+                    break;
+                }
                 if (++slot == BULK_SCHED_DEPTH) { slot = 0; phase ^= 1u; }
             }
         }
