@@ -48,6 +48,9 @@ def _load():
             ctypes.c_double, ctypes.c_double, ctypes.c_int32,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
         ]
+        lib.oracle_outer_sync_ex.restype = ctypes.c_int
+        lib.oracle_outer_sync_ex.argtypes = lib.oracle_outer_sync.argtypes + [ctypes.c_void_p,
+                                                                              ctypes.c_void_p]
         lib.oracle_max_threads.restype = ctypes.c_int32
         lib.oracle_max_threads.argtypes = []
         _lib = lib
@@ -60,13 +63,15 @@ def max_threads() -> int:
 
 def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, paths,
                path_dtype, outer_lr, outer_momentum, path_weights=None, reported=None,
-               num_threads=1):
+               num_threads=1, module_scale=None, level_sync=None):
     """Run one outer synchronisation in place on host arrays.
 
     theta, momentum: contiguous float32 numpy arrays of sum_l K_l*N_l elements (level, module,
     element order).  paths: list of P contiguous numpy arrays, float32 for ``F32`` or uint16
     (raw bf16 bits) for ``BF16``, each of sum_l N_l elements.  path_to_module: int array [P, L].
     path_weights: None (uniform) or [P] float32.  reported: None (all) or [P] of 0/1.
+    module_scale: None or [sum_l K_l] factors on the modules' outer gradients (level-major).
+    level_sync: None or [L] of 0/1, 0 = the level is left untouched.
     """
     lib = _load()
     K = np.ascontiguousarray(modules_per_level, dtype=np.int32)
@@ -92,13 +97,23 @@ def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, 
     if reported is not None:
         r = np.ascontiguousarray(reported, dtype=np.uint8)
         assert r.shape == (P,)
-    rc = lib.oracle_outer_sync(
+    sc = None
+    if module_scale is not None:
+        sc = np.ascontiguousarray(module_scale, dtype=np.float64)
+        assert sc.shape == (int(K.sum()),)
+    ls = None
+    if level_sync is not None:
+        ls = np.ascontiguousarray(level_sync, dtype=np.uint8)
+        assert ls.shape == (L,)
+    rc = lib.oracle_outer_sync_ex(
         L, K.ctypes.data, N.ctypes.data, P, table.ctypes.data,
         w.ctypes.data if w is not None else None,
         r.ctypes.data if r is not None else None,
         float(outer_lr), float(outer_momentum), int(path_dtype),
         theta.ctypes.data, momentum.ctypes.data, ctypes.cast(ptrs, ctypes.c_void_p),
         int(num_threads),
+        sc.ctypes.data if sc is not None else None,
+        ls.ctypes.data if ls is not None else None,
     )
     if rc != 0:
         raise ValueError("oracle_outer_sync rejected its arguments")

@@ -24,6 +24,15 @@
  *   4. every path of S(l,e), reporting or not, receives cast(theta')
  *      (Section 2.5: the new global vector is re-dispatched to all workers).
  *
+ * Two options of Section 2.7 / Section 4.1, off by default:
+ *   - module_scale: the outer gradient of module (l,e) is multiplied by s(l,e) before the
+ *     optimiser step, Delta <- s * Delta ("Outer Gradient Norm Rescaling": the paper rescales
+ *     by the square root of the number of paths through the module; the caller supplies s, so
+ *     whether that means sqrt(P) or 1/sqrt(P) is the caller's reading).
+ *   - level_sync: a level flagged 0 takes no part in the exchange (Section 4.1 keeps some
+ *     blocks of the path-specific models local to their path): theta, momentum and every copy
+ *     of its modules are left untouched.
+ *
  * Arithmetic: steps 1-3 in double, theta' and m' rounded once to float;
  * a bf16 path copy receives round-to-nearest-even of that float.
  * Loop order: module, element, contributor (ascending path id).
@@ -98,14 +107,18 @@ static void write_copy(void *buf, int dtype, int64_t idx, float v)
  *  path_ptrs           [P] pointers; copy i holds its L modules concatenated in level order
  *  num_threads         OpenMP threads for the element loop (elements are independent)
  *
+ *  module_scale        [sum_l K_l] factor on each module's outer gradient, level-major, or NULL = 1
+ *  level_sync          [L] 0 = leave the level untouched, or NULL = every level is synchronised
+ *
  * Returns 0, or -1 on an invalid argument.
  */
-int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
-                      const int64_t *level_numel, int32_t num_paths,
-                      const int32_t *path_to_module, const float *path_weights,
-                      const uint8_t *reported, double outer_lr, double outer_momentum,
-                      int32_t path_dtype, float *theta, float *momentum,
-                      void *const *path_ptrs, int32_t num_threads)
+int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
+                         const int64_t *level_numel, int32_t num_paths,
+                         const int32_t *path_to_module, const float *path_weights,
+                         const uint8_t *reported, double outer_lr, double outer_momentum,
+                         int32_t path_dtype, float *theta, float *momentum,
+                         void *const *path_ptrs, int32_t num_threads,
+                         const double *module_scale, const uint8_t *level_sync)
 {
     if (num_levels < 1 || num_paths < 1 || !modules_per_level || !level_numel ||
         !path_to_module || !theta || !momentum || !path_ptrs)
@@ -132,9 +145,17 @@ int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
 
     int64_t module_base = 0;  /* offset of module (l,e) inside theta / momentum */
     int64_t level_base = 0;   /* offset of level l inside one path copy */
+    int32_t module_index = 0; /* level-major index of module (l,e) */
     for (int32_t l = 0; l < num_levels; ++l) {
         const int64_t n = level_numel[l];
-        for (int32_t e = 0; e < modules_per_level[l]; ++e) {
+        if (level_sync && !level_sync[l]) {  /* level not communicated: nothing is touched */
+            module_base += n * modules_per_level[l];
+            module_index += modules_per_level[l];
+            level_base += n;
+            continue;
+        }
+        for (int32_t e = 0; e < modules_per_level[l]; ++e, ++module_index) {
+            const double scale = module_scale ? module_scale[module_index] : 1.0;
             /* S(l,e) and R(l,e) by a linear scan of the table, ascending path id */
             int32_t n_members = 0, n_reporters = 0;
             double total_weight = 0.0;
@@ -168,6 +189,7 @@ int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
                         double x = read_copy(path_ptrs[reporters[r]], path_dtype, level_base + k);
                         delta += alpha[r] * (t0 - x);
                     }
+                    delta *= scale;
                     const double m1 = outer_momentum * (double)mo[k] + delta;
                     const double t1 = t0 - outer_lr * (delta + outer_momentum * m1);
                     mo[k] = (float)m1;
@@ -183,6 +205,18 @@ int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
     }
     free(members); free(reporters); free(alpha);
     return 0;
+}
+
+int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
+                      const int64_t *level_numel, int32_t num_paths,
+                      const int32_t *path_to_module, const float *path_weights,
+                      const uint8_t *reported, double outer_lr, double outer_momentum,
+                      int32_t path_dtype, float *theta, float *momentum,
+                      void *const *path_ptrs, int32_t num_threads)
+{
+    return oracle_outer_sync_ex(num_levels, modules_per_level, level_numel, num_paths,
+                                path_to_module, path_weights, reported, outer_lr, outer_momentum,
+                                path_dtype, theta, momentum, path_ptrs, num_threads, NULL, NULL);
 }
 
 /* number of OpenMP threads the element loop can use on this host (1 without OpenMP) */

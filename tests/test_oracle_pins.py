@@ -440,3 +440,49 @@ def test_rejects_a_table_entry_out_of_range():
     with pytest.raises(ValueError):
         oracle.outer_sync(cfg.modules_per_level, cfg.level_numel, table, th, th.copy(),
                           [np.zeros(8, np.float32) for _ in range(2)], oracle.F32, LR, MU)
+
+
+# ---------------------------------------------------------------------------- Section 2.7 options
+
+def test_module_scale_multiplies_the_outer_gradient():
+    """Delta <- s * Delta: with m = 0 the new momentum is s times the unscaled one; with lr = 1,
+    mu = 0 theta' = theta - s * (theta - mean); s = 0 leaves theta and only decays momentum."""
+    cfg = tiny_cfg((1, 2, 2), (6, 5, 7), seed=21)
+    pr = synth.make_problem(cfg)
+    th, mo, ps = helpers.host_copy(pr)
+    scale = np.array([2.0, 0.5, 4.0, 1.0, 0.0])          # one per module, level-major
+    _, base_mo, _ = helpers.run_oracle(cfg, pr.table, th, mo, ps)
+    got_th, got_mo, _ = helpers.run_oracle(cfg, pr.table, th, mo, ps, module_scale=scale)
+    mean_th, _, _ = helpers.run_oracle(cfg, pr.table, th, mo, ps, lr=1.0, mu=0.0, module_scale=scale)
+    for idx, (l, e, ts, psl) in enumerate(module_slices(cfg)):
+        np.testing.assert_allclose(got_mo[ts], scale[idx] * base_mo[ts].astype(np.float64),
+                                   rtol=2e-7, atol=0)
+        S = [i for i in range(cfg.num_paths) if pr.table[i, l] == e]
+        mean = np.mean(np.stack([ps[i][psl].astype(np.float64) for i in S]), axis=0)
+        want = th[ts] - scale[idx] * (th[ts].astype(np.float64) - mean)
+        assert np.all(np.abs(mean_th[ts] - want) <= one_ulp(want))
+    last = module_slices(cfg)[-1][2]
+    np.testing.assert_array_equal(got_th[last], th[last])   # s = 0, m = 0: nothing moves
+    ones = helpers.run_oracle(cfg, pr.table, th, mo, ps, module_scale=np.ones(5))
+    plain = helpers.run_oracle(cfg, pr.table, th, mo, ps)
+    np.testing.assert_array_equal(ones[0], plain[0])
+    np.testing.assert_array_equal(ones[1], plain[1])
+
+
+def test_levels_flagged_as_not_communicated_are_left_untouched():
+    cfg = tiny_cfg((1, 2, 2), (6, 5, 7), "bf16", momentum_std=1e-2, seed=22)
+    pr = synth.make_problem(cfg)
+    th, mo, ps = helpers.host_copy(pr)
+    flags = np.array([1, 0, 1], dtype=np.uint8)
+    got_th, got_mo, got_ps = helpers.run_oracle(cfg, pr.table, th, mo, ps, level_sync=flags)
+    full_th, full_mo, full_ps = helpers.run_oracle(cfg, pr.table, th, mo, ps)
+    skipped = slice(6, 16)          # the two level-2 modules of 5 parameters each
+    np.testing.assert_array_equal(got_th[skipped], th[skipped])
+    np.testing.assert_array_equal(got_mo[skipped], mo[skipped])
+    for i in range(cfg.num_paths):
+        np.testing.assert_array_equal(got_ps[i][6:11], ps[i][6:11])       # copies keep their own values
+        np.testing.assert_array_equal(got_ps[i][:6], full_ps[i][:6])
+        np.testing.assert_array_equal(got_ps[i][11:], full_ps[i][11:])
+    np.testing.assert_array_equal(got_th[:6], full_th[:6])
+    np.testing.assert_array_equal(got_th[16:], full_th[16:])
+    np.testing.assert_array_equal(got_mo[16:], full_mo[16:])
