@@ -136,6 +136,22 @@ int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_h
 /* Replace the raw per-path weights (host [P], or NULL = uniform).  Section 2.7. */
 int dipaco_set_weights(dipaco_ctx *ctx, const float *path_weights);
 
+/*
+ * Outer gradient norm rescaling (Section 2.7): the finished outer gradient of module (l,e) is
+ * multiplied by module_scale[(l,e)] before the optimiser step, Delta <- s * Delta.  host
+ * [sum_l K_l], level-major, finite; NULL = no rescaling.  The paper rescales by the square root
+ * of the number of paths through the module; the factor itself (sqrt(P) or its inverse) is the
+ * caller's to supply.  A factor of exactly 1 leaves the result bit-identical.
+ */
+int dipaco_set_module_scale(dipaco_ctx *ctx, const float *module_scale);
+
+/*
+ * Levels that take no part in the exchange (Section 4.1: in the models with path-specific
+ * modules some blocks stay local to their path): host [L], 0 = theta, momentum and every copy
+ * of the level's modules are left untouched; NULL = every level is synchronised.
+ */
+int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync);
+
 /* Choose the kernel family (DIPACO_KERNEL_*); all families give bitwise identical results. */
 int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
 

@@ -39,7 +39,8 @@ EXPORTS = [
     "dipaco_outer_sync_host", "dipaco_set_weights", "dipaco_set_kernel", "dipaco_set_tuning",
     "dipaco_device_status", "dipaco_launch_count", "dipaco_plan_module", "dipaco_plan_offsets",
     "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
-    "dipaco_set_host_unit_bytes", "dipaco_plan_traffic",
+    "dipaco_set_host_unit_bytes", "dipaco_plan_traffic", "dipaco_set_module_scale",
+    "dipaco_set_level_sync",
 ]
 
 _lib = None
@@ -73,6 +74,8 @@ def load() -> ctypes.CDLL:
     lib.dipaco_sync_end.argtypes = [vp]
     lib.dipaco_outer_sync_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dipaco_set_weights.argtypes = [vp, vp]
+    lib.dipaco_set_module_scale.argtypes = [vp, vp]
+    lib.dipaco_set_level_sync.argtypes = [vp, vp]
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32]
     lib.dipaco_device_status.argtypes = [vp]
@@ -188,6 +191,16 @@ def dipaco_outer_sync_host(ctx, theta_host_ptr, momentum_host_ptr, path_host_ptr
 def dipaco_set_weights(ctx, path_weights) -> None:
     w = None if path_weights is None else np.ascontiguousarray(path_weights, dtype=np.float32)
     _check(load().dipaco_set_weights(ctx, _np_ptr(w)), "dipaco_set_weights")
+
+
+def dipaco_set_module_scale(ctx, module_scale) -> None:
+    sc = None if module_scale is None else np.ascontiguousarray(module_scale, dtype=np.float32)
+    _check(load().dipaco_set_module_scale(ctx, _np_ptr(sc)), "dipaco_set_module_scale")
+
+
+def dipaco_set_level_sync(ctx, level_sync) -> None:
+    ls = None if level_sync is None else np.ascontiguousarray(level_sync, dtype=np.uint8)
+    _check(load().dipaco_set_level_sync(ctx, _np_ptr(ls)), "dipaco_set_level_sync")
 
 
 def dipaco_set_kernel(ctx, kernel: int) -> None:

@@ -172,7 +172,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         pd.theta_off = m.theta_off;
         pd.partial_off = m.partial_off >= 0 ? m.partial_off : 0;
         pd.flags = sp.flags;
-        pd.pad = 0;
+        pd.scale = sp.scale;
         pd.item_first = 0;
         pd.tiles_per_item = 1;
         pd.bulk_tiles = 0;
@@ -554,6 +554,30 @@ int dipaco_set_weights(dipaco_ctx *ctx, const float *path_weights)
     } else {
         ctx->grid.weights.clear();
     }
+    return DIPACO_OK;
+}
+
+int dipaco_set_module_scale(dipaco_ctx *ctx, const float *module_scale)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (module_scale) {
+        const size_t n = ctx->grid.modules.size();
+        for (size_t i = 0; i < n; ++i)
+            if (!std::isfinite(module_scale[i])) return DIPACO_EINVAL;
+        ctx->grid.module_scale.assign(module_scale, module_scale + n);
+    } else {
+        ctx->grid.module_scale.clear();
+    }
+    return DIPACO_OK;
+}
+
+int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync)
+{
+    if (!ctx) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (level_sync) ctx->grid.level_sync.assign(level_sync, level_sync + ctx->grid.L);
+    else ctx->grid.level_sync.clear();
     return DIPACO_OK;
 }
 

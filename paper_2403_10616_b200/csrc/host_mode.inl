@@ -120,7 +120,7 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
     for (size_t id = 0; id < g.modules.size(); ++id) {
         const ModuleGeom &m = g.modules[id];
         const ModuleCoeffs &mc = ctx->coeffs[id];
-        if (m.members.empty() || m.numel == 0) continue;
+        if (m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
         const size_t ncon = mc.contributors.size();
         // elements per unit: every reporting copy's piece must fit the input buffer
         // and a unit uploads at most HOST_UNIT_BYTES so that the pipeline fills and drains quickly
@@ -174,6 +174,7 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
                 PassSpec sp;
                 sp.module = (int)id;
                 sp.flags = mc.update ? PASS_UPDATE : 0;
+                sp.scale = g.scale_of(id);
                 sp.contributors = mc.contributors;
                 sp.coeff = mc.coeff;
                 sp.begin = a;

@@ -28,7 +28,7 @@ struct PassDev {
     // [item_first, item_first + ceil(bulk_tiles / tiles_per_item)), each a run of full tiles
     int item_first;
     int tiles_per_item;
-    int pad;
+    float scale;  // factor on the finished outer gradient (Section 2.7, norm rescaling); 1 = none
     long long bulk_tiles;
     long long bulk_begin;  // element range [bulk_begin, bulk_end) of the module that the bulk-copy
     long long bulk_end;    // kernel covers: whole 16-byte units of path data; the last tile of the
@@ -74,10 +74,11 @@ __device__ __forceinline__ float sync_accumulate(float acc, float c, float theta
     return __fmaf_rn(c, __fsub_rn(theta, x), acc);
 }
 
-__device__ __forceinline__ void sync_nesterov(float theta, float m, float delta, float lr, float mu,
-                                              float &theta_new, float &m_new)
+__device__ __forceinline__ void sync_nesterov(float theta, float m, float sum, float scale, float lr,
+                                              float mu, float &theta_new, float &m_new)
 {
-    // m' = mu*m + Delta ; theta' = theta - lr*(Delta + mu*m')
+    // Delta = scale * sum ; m' = mu*m + Delta ; theta' = theta - lr*(Delta + mu*m')
+    const float delta = __fmul_rn(scale, sum);  // exact when scale == 1
     m_new = __fmaf_rn(mu, m, delta);
     const float g = __fmaf_rn(mu, m_new, delta);
     theta_new = __fmaf_rn(-lr, g, theta);
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
 #pragma unroll
                 for (int v = 0; v < VEC; ++v) {
                     float t1, m1;
-                    sync_nesterov(th[v], mo[v], acc[v], p.lr, p.mu, t1, m1);
+                    sync_nesterov(th[v], mo[v], acc[v], pass.scale, p.lr, p.mu, t1, m1);
                     th[v] = t1;
                     mo[v] = m1;
                 }
@@ -735,8 +736,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                         float m1[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            sync_nesterov(th[u * UE + v + i], mo[i], acc[u * UE + v + i], p.lr, p.mu,
-                                          th[u * UE + v + i], m1[i]);
+                            sync_nesterov(th[u * UE + v + i], mo[i], acc[u * UE + v + i], pass.scale, p.lr,
+                                          p.mu, th[u * UE + v + i], m1[i]);
                         *reinterpret_cast<float4 *>(mo_tile + e0 + v) =
                             make_float4(m1[0], m1[1], m1[2], m1[3]);
                         *reinterpret_cast<float4 *>(th_tile + e0 + v) =

@@ -32,6 +32,8 @@ struct Grid {
     std::vector<int64_t> N;
     std::vector<int> table;          // [P*L]
     std::vector<float> weights;      // [P] or empty = uniform
+    std::vector<float> module_scale; // [modules] factor on the outer gradient, empty = 1
+    std::vector<uint8_t> level_sync; // [L] 0 = level takes no part in the exchange, empty = all do
     std::vector<int> level_first;    // module id of (l,0)
     std::vector<ModuleGeom> modules; // level-major
     int64_t module_params = 0, params_per_path = 0;
@@ -39,6 +41,8 @@ struct Grid {
     int64_t scratch_elems = 0;
 
     int module_id(int l, int e) const { return level_first[l] + e; }
+    bool synced(const ModuleGeom &m) const { return level_sync.empty() || level_sync[(size_t)m.level]; }
+    float scale_of(size_t id) const { return module_scale.empty() ? 1.0f : module_scale[id]; }
     int chunk_of(int path) const { return chunk_paths > 0 ? path / chunk_paths : 0; }
 };
 
@@ -138,6 +142,7 @@ struct PassSpec {
     std::vector<float> coeff;
     std::vector<int> members;      // path ids written in this launch
     int64_t begin = 0, end = -1;   // element range of the module ([0, numel) when end < 0)
+    float scale = 1.0f;            // factor on the finished outer gradient (used with PASS_UPDATE)
 };
 
 // Resident mode: one launch covers every module completely.
@@ -147,9 +152,10 @@ inline void plan_resident(const Grid &g, const std::vector<ModuleCoeffs> &mc,
     out.clear();
     for (size_t id = 0; id < g.modules.size(); ++id) {
         const ModuleGeom &m = g.modules[id];
-        if (m.members.empty() || m.numel == 0) continue;
+        if (m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
         PassSpec p;
         p.module = (int)id;
+        p.scale = g.scale_of(id);
         p.flags = mc[id].update ? PASS_UPDATE : 0;
         p.contributors = mc[id].contributors;
         p.coeff = mc[id].coeff;
@@ -166,11 +172,12 @@ inline void plan_accumulate(const Grid &g, const std::vector<ModuleCoeffs> &mc, 
     for (size_t id = 0; id < g.modules.size(); ++id) {
         const ModuleGeom &m = g.modules[id];
         const ModuleCoeffs &k = mc[id];
-        if (!k.update || m.numel == 0) continue;
+        if (!k.update || m.numel == 0 || !g.synced(m)) continue;
         const int first = g.chunk_of(k.contributors.front());
         const int last = g.chunk_of(k.contributors.back());
         PassSpec p;
         p.module = (int)id;
+        p.scale = g.scale_of(id);
         for (size_t j = 0; j < k.contributors.size(); ++j)
             if (g.chunk_of(k.contributors[j]) == c) {
                 p.contributors.push_back(k.contributors[j]);
@@ -198,7 +205,7 @@ inline void plan_writeback(const Grid &g, const std::vector<ModuleCoeffs> &mc, i
     for (size_t id = 0; id < g.modules.size(); ++id) {
         const ModuleGeom &m = g.modules[id];
         const ModuleCoeffs &k = mc[id];
-        if (m.numel == 0) continue;
+        if (m.numel == 0 || !g.synced(m)) continue;
         if (skip_final && k.update && g.chunk_of(k.contributors.back()) == c) continue;
         PassSpec p;
         p.module = (int)id;

@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(256) static_accumulate_kernel(StaticAccumulate
         if (a.flags & KPASS_PARTIAL_OUT) a.partial[k] = acc;
         if (a.flags & KPASS_UPDATE) {
             float t1, m1;
-            sync_nesterov(th, a.momentum[k], acc, a.lr, a.mu, t1, m1);
+            sync_nesterov(th, a.momentum[k], acc, 1.0f, a.lr, a.mu, t1, m1);
             a.theta[k] = t1;
             a.momentum[k] = m1;
         }

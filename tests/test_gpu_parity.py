@@ -341,3 +341,44 @@ def test_host_buffers_entry_point_matches_the_oracle(name, pinned):
     state = (dev.theta.to(DEV), dev.momentum.to(DEV), [p.to(DEV) for p in dev.paths])
     run_gpu(pr, state)
     assert_states_bitwise_equal((theta.to(DEV), momentum.to(DEV), [p.to(DEV) for p in paths]), state)
+
+
+@pytest.mark.parametrize("mode", ["resident", "chunked", "host"])
+def test_gradient_rescaling_and_levels_kept_local(mode):
+    """Section 2.7 rescaling (here sqrt of the number of paths through each module) and a level
+    that takes no part in the exchange, against the oracle, in every mode."""
+    base = synth.CONFIGS["grid16x16-masked"]
+    cfg = base.scaled((2 * 4096 + 72, 4096 + 8, 3 * 4096 + 1003))
+    pr = synth.make_problem(cfg, "cpu" if mode == "host" else DEV)
+    before = host_state(clone_problem(pr))
+    scale = np.concatenate([[np.sqrt(256.0)], np.full(16, np.sqrt(16.0)),
+                            np.sqrt(np.arange(1, 17))]).astype(np.float32)
+    flags = np.array([1, 0, 1], dtype=np.uint8)
+    theta, momentum, paths = clone_problem(pr)
+    ctx = make_ctx(pr, chunk_paths=0 if mode == "resident" else 32)
+    B.dipaco_set_module_scale(ctx, scale)
+    B.dipaco_set_level_sync(ctx, flags)
+    ptrs = [p.data_ptr() for p in paths]
+    if mode == "host":
+        B.dipaco_outer_sync_host(ctx, theta.data_ptr(), momentum.data_ptr(), ptrs, pr.reported)
+    else:
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), ptrs, pr.reported)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    B.dipaco_destroy(ctx)
+    want_th, want_mo, want_ps = helpers.run_oracle(cfg, pr.table, *before, pr.weights, pr.reported,
+                                                   num_threads=8, module_scale=scale.astype(np.float64),
+                                                   level_sync=flags)
+    got_th, got_mo = helpers.tensor_to_numpy(theta), helpers.tensor_to_numpy(momentum)
+    for got, want in ((got_th, want_th), (got_mo, want_mo)):
+        err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+        assert np.all(err <= 1e-6 * (1.0 + np.abs(want.astype(np.float64))))
+    n0, n1, n2 = cfg.level_numel
+    # the level kept local is bitwise untouched everywhere
+    np.testing.assert_array_equal(got_th[n0:n0 + 16 * n1], before[0][n0:n0 + 16 * n1])
+    np.testing.assert_array_equal(got_mo[n0:n0 + 16 * n1], before[1][n0:n0 + 16 * n1])
+    for i, p in enumerate(paths):
+        got = helpers.tensor_to_numpy(p)
+        np.testing.assert_array_equal(got[n0:n0 + n1], before[2][i][n0:n0 + n1])
+        assert_bf16_close(got[:n0], want_ps[i][:n0])
+        assert_bf16_close(got[n0 + n1:], want_ps[i][n0 + n1:])
+    assert not np.array_equal(got_th[:n0], before[0][:n0])
