@@ -36,8 +36,8 @@ REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the referen
 # by the algorithmic bytes of that launch.  Traffic grows with the number of tiles, so the full-size
 # figure is this ratio times the algorithmic bytes.  Only valid for the kernel source it was taken
 # from: the digest below is checked and "traffic" is null after any change to the kernels.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9912
-NCU_CAPTURE_KERNELS_SHA256 = "unset"
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9918
+NCU_CAPTURE_KERNELS_SHA256 = "98d96b4add4d32686e689781009bc1b4ccf6022105b8f0003f5f5bf966e0cd8d"
 
 
 def kernels_digest():
