@@ -61,6 +61,7 @@ def parse_args():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--units", type=int, default=0)
+    ap.add_argument("--io-slots", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-chunked", action="store_true")
@@ -327,7 +328,7 @@ def run_ours(args):
                               np.float32(cfg.outer_lr), np.float32(cfg.outer_momentum), code,
                               chunk_paths, local)
         B.dipaco_set_kernel(ctx, kernel)
-        B.dipaco_set_tuning(ctx, args.ctas_per_sm, args.stages, args.units)
+        B.dipaco_set_tuning(ctx, args.ctas_per_sm, args.stages, args.units, args.io_slots)
         return ctx
 
     # ---- resident one-pass mode: the headline value

@@ -156,13 +156,15 @@ int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync);
 int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
 
 /*
- * Tuning of the bulk-copy kernel: persistent CTAs per SM (1..8), pipeline depth in tiles (2..32)
- * and 16-byte units of path data per compute thread and tile (1, 2 or 4; the tile is
- * 256 threads * units * 16 bytes).  0 keeps a value.  A depth that does not fit the shared
- * memory of the chosen layout is rejected with DIPACO_EINVAL and nothing changes.
+ * Tuning of the bulk-copy kernel: persistent CTAs per SM (1..8), pipeline depth in tiles (2..32),
+ * 16-byte units of path data per compute thread and tile (1, 2 or 4; the tile is
+ * 256 threads * units * 16 bytes) and the number of theta/momentum/result tile buffers (2..4;
+ * more of them help modules with few contributors).  0 keeps a value.  A depth that does not fit
+ * the shared memory of the chosen layout is rejected with DIPACO_EINVAL and nothing changes;
+ * result buffers beyond two are dropped at launch if they would leave fewer than 6 stages.
  */
 int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
-                      int32_t units_per_thread);
+                      int32_t units_per_thread, int32_t io_slots);
 
 /*
  * Tuning of dipaco_outer_sync_host: the most bytes of path data one streamed unit uploads

@@ -77,7 +77,7 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_module_scale.argtypes = [vp, vp]
     lib.dipaco_set_level_sync.argtypes = [vp, vp]
     lib.dipaco_set_kernel.argtypes = [vp, i32]
-    lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32]
+    lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32, i32]
     lib.dipaco_device_status.argtypes = [vp]
     lib.dipaco_set_host_unit_bytes.argtypes = [vp, i64]
     lib.dipaco_launch_count.argtypes = [vp]
@@ -207,9 +207,9 @@ def dipaco_set_kernel(ctx, kernel: int) -> None:
     _check(load().dipaco_set_kernel(ctx, int(kernel)), "dipaco_set_kernel")
 
 
-def dipaco_set_tuning(ctx, ctas_per_sm=0, stages=0, units_per_thread=0) -> None:
-    _check(load().dipaco_set_tuning(ctx, int(ctas_per_sm), int(stages), int(units_per_thread)),
-           "dipaco_set_tuning")
+def dipaco_set_tuning(ctx, ctas_per_sm=0, stages=0, units_per_thread=0, io_slots=0) -> None:
+    _check(load().dipaco_set_tuning(ctx, int(ctas_per_sm), int(stages), int(units_per_thread),
+                                    int(io_slots)), "dipaco_set_tuning")
 
 
 def dipaco_set_host_unit_bytes(ctx, nbytes: int) -> None:

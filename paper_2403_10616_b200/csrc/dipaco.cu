@@ -55,6 +55,7 @@ struct dipaco_ctx {
     int sm_count = 0;
     int kernel = DIPACO_KERNEL_AUTO;
     int ctas_per_sm = 1, stages = 10, units = 2;  // bulk-copy kernel tuning (measured on B200)
+    int io_slots = 3;                            // buffers of theta/momentum/result tiles
     int64_t launches = 0;
     int64_t host_unit_bytes = (int64_t)1 << 40;  // upload size cap of one unit in host mode
 
@@ -116,22 +117,22 @@ int64_t tile_elems(const dipaco_ctx *ctx)
 }
 
 // Shared memory of one bulk-kernel CTA for a given depth.
-size_t bulk_smem_bytes(const dipaco_ctx *ctx, int stages, int io_arrays)
+size_t bulk_smem_bytes(const dipaco_ctx *ctx, int stages, int io_arrays, int io_slots)
 {
     const size_t tile = (size_t)tile_elems(ctx);
     const size_t stage = tile * ctx->elem_size;
-    size_t bytes = (size_t)stages * stage + (size_t)2 * io_arrays * tile * 4;
-    if (ctx->elem_size != 4) bytes += 2 * stage;
+    size_t bytes = (size_t)stages * stage + (size_t)io_slots * io_arrays * tile * 4;
+    if (ctx->elem_size != 4) bytes += (size_t)io_slots * stage;
     return bytes + sizeof(BulkShared) + 128;
 }
 
-int pick_stages(const dipaco_ctx *ctx, int io_arrays)
+int pick_stages(const dipaco_ctx *ctx, int io_arrays, int io_slots)
 {
     const size_t budget =
         std::min(SMEM_LIMIT, SMEM_PER_SM / (size_t)ctx->ctas_per_sm - 2 * SMEM_CTA_RESERVE);
     int best = 0;
     for (int s = 2; s <= BULK_MAX_STAGES; ++s)
-        if (bulk_smem_bytes(ctx, s, io_arrays) <= budget) best = s;
+        if (bulk_smem_bytes(ctx, s, io_arrays, io_slots) <= budget) best = s;
     if (ctx->stages > 0) return ctx->stages <= best ? ctx->stages : best;
     return best;
 }
@@ -335,7 +336,7 @@ int upload_blob(dipaco_ctx *ctx, const std::vector<unsigned char> &blob, cudaStr
 }
 
 template <typename PathT, int NU>
-int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages, int io_arrays,
+int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages, int io_arrays, int io_slots,
                   size_t smem, int attr_row, int attr_col, cudaStream_t stream)
 {
     if (!ctx->smem_attr_set[attr_row][attr_col]) {
@@ -345,25 +346,28 @@ int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages,
             return DIPACO_ECUDA;
         ctx->smem_attr_set[attr_row][attr_col] = true;
     }
-    sync_bulk_kernel<PathT, NU><<<ctas, BULK_THREADS, smem, stream>>>(lp, stages, io_arrays);
+    sync_bulk_kernel<PathT, NU><<<ctas, BULK_THREADS, smem, stream>>>(lp, stages, io_arrays, io_slots);
     return cudaGetLastError() == cudaSuccess ? DIPACO_OK : DIPACO_ECUDA;
 }
 
 int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays, cudaStream_t stream)
 {
-    const int stages = pick_stages(ctx, io_arrays);
+    // more result buffers only while the copy ring keeps a useful depth
+    int io_slots = ctx->io_slots;
+    while (io_slots > 2 && pick_stages(ctx, io_arrays, io_slots) < 6) --io_slots;
+    const int stages = pick_stages(ctx, io_arrays, io_slots);
     if (stages < 2) return DIPACO_EINVAL;
-    const size_t smem = bulk_smem_bytes(ctx, stages, io_arrays);
+    const size_t smem = bulk_smem_bytes(ctx, stages, io_arrays, io_slots);
     const int nu = tile_units(ctx);
     const int col = nu == 1 ? 0 : (nu == 2 ? 1 : 2);
     if (ctx->dtype == DIPACO_BF16) {
-        if (nu == 1) return launch_bulk_t<__nv_bfloat16, 1>(ctx, lp, ctas, stages, io_arrays, smem, 1, col, stream);
-        if (nu == 2) return launch_bulk_t<__nv_bfloat16, 2>(ctx, lp, ctas, stages, io_arrays, smem, 1, col, stream);
-        return launch_bulk_t<__nv_bfloat16, 4>(ctx, lp, ctas, stages, io_arrays, smem, 1, col, stream);
+        if (nu == 1) return launch_bulk_t<__nv_bfloat16, 1>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
+        if (nu == 2) return launch_bulk_t<__nv_bfloat16, 2>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
+        return launch_bulk_t<__nv_bfloat16, 4>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
     }
-    if (nu == 1) return launch_bulk_t<float, 1>(ctx, lp, ctas, stages, io_arrays, smem, 0, col, stream);
-    if (nu == 2) return launch_bulk_t<float, 2>(ctx, lp, ctas, stages, io_arrays, smem, 0, col, stream);
-    return launch_bulk_t<float, 4>(ctx, lp, ctas, stages, io_arrays, smem, 0, col, stream);
+    if (nu == 1) return launch_bulk_t<float, 1>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 0, col, stream);
+    if (nu == 2) return launch_bulk_t<float, 2>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 0, col, stream);
+    return launch_bulk_t<float, 4>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 0, col, stream);
 }
 
 int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *momentum,
@@ -589,7 +593,8 @@ int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel)
     return DIPACO_OK;
 }
 
-int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int32_t units_per_thread)
+int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int32_t units_per_thread,
+                      int32_t io_slots)
 {
     if (!ctx) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
@@ -597,13 +602,14 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
         return DIPACO_EINVAL;
     if (units_per_thread != 0 && units_per_thread != 1 && units_per_thread != 2 && units_per_thread != 4)
         return DIPACO_EINVAL;
+    if (io_slots != 0 && (io_slots < 2 || io_slots > BULK_MAX_IO_SLOTS)) return DIPACO_EINVAL;
     const int old_ctas = ctx->ctas_per_sm, old_units = ctx->units, old_stages = ctx->stages;
     if (ctas_per_sm) ctx->ctas_per_sm = ctas_per_sm;
     if (units_per_thread) ctx->units = units_per_thread;
     ctx->stages = 0;
     // chunked contexts stage a third fp32 tile (the partial sum) per buffer
     const int io_arrays = ctx->grid.num_chunks > 1 ? 3 : 2;
-    const bool fits = pick_stages(ctx, io_arrays) >= 2 && (!stages || stages <= pick_stages(ctx, io_arrays));
+    const bool fits = pick_stages(ctx, io_arrays, 2) >= 2 && (!stages || stages <= pick_stages(ctx, io_arrays, 2));
     if (!fits) {
         ctx->ctas_per_sm = old_ctas;
         ctx->units = old_units;
@@ -611,6 +617,7 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
         return DIPACO_EINVAL;
     }
     ctx->stages = stages ? stages : old_stages;
+    if (io_slots) ctx->io_slots = io_slots;
     return DIPACO_OK;
 }
 

@@ -370,6 +370,7 @@ constexpr int BULK_COMPUTE_THREADS = BULK_COMPUTE_WARPS * 32;
 constexpr int BULK_THREADS = BULK_COMPUTE_THREADS + 96;  // + load, store and scheduler warps
 constexpr int BULK_MAX_STAGES = 32;
 constexpr int BULK_SCHED_DEPTH = 4;
+constexpr int BULK_MAX_IO_SLOTS = 4;  // buffers of theta/momentum/partial/result tiles
 constexpr int BULK_ITEM_READERS = BULK_COMPUTE_WARPS + 2;  // warps that consume every work item
 constexpr unsigned long long BULK_WAIT_LIMIT_NS = 4000000000ull;  // every wait gives up after 4 s
 
@@ -392,9 +393,9 @@ __device__ __forceinline__ bool bounded_wait(uint64_t *bar, unsigned parity, int
 struct BulkShared {
     uint64_t full[BULK_MAX_STAGES];   // ring slot filled by a bulk load
     uint64_t empty[BULK_MAX_STAGES];  // ring slot released by the compute warps
-    uint64_t io_full[2];              // theta / momentum / partial tiles loaded
-    uint64_t io_empty[2];             // result tiles drained by the store warp
-    uint64_t out_ready[2];            // compute warps finished writing the result tiles
+    uint64_t io_full[BULK_MAX_IO_SLOTS];    // theta / momentum / partial tiles loaded
+    uint64_t io_empty[BULK_MAX_IO_SLOTS];   // result tiles drained by the store warp
+    uint64_t out_ready[BULK_MAX_IO_SLOTS];  // compute warps finished writing the result tiles
     uint64_t sched_full[BULK_SCHED_DEPTH];   // a work item was published by the scheduler warp
     uint64_t sched_empty[BULK_SCHED_DEPTH];  // all ten consumer warps have read it
     long long sched_begin[BULK_SCHED_DEPTH], sched_end[BULK_SCHED_DEPTH];
@@ -467,7 +468,7 @@ struct ItemWalk {
 // NU = 16-byte units of path data per compute thread and tile; tile = 256 * NU * UE elements.
 template <typename PathT, int NU>
 __global__ void __launch_bounds__(BULK_THREADS, 1)
-sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
+sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
 {
     constexpr int UE = Unit<PathT>::UE;
     constexpr int EPT = UE * NU;                         // elements per compute thread
@@ -477,11 +478,12 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
     constexpr bool NEED_CAST_TILE = sizeof(PathT) != 4;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    // layout: ring | io[2][io_arrays] fp32 tiles | cast tile[2] (bf16 only) | BulkShared
+    // layout: ring | io[io_slots][io_arrays] fp32 tiles | cast tile[io_slots] (bf16 only) | BulkShared
     unsigned char *ring = smem_raw;
     unsigned char *io = ring + (size_t)stages * STAGE_BYTES;
-    unsigned char *cast_tiles = io + (size_t)2 * io_arrays * F32_TILE_BYTES;
-    BulkShared *sh = reinterpret_cast<BulkShared *>(cast_tiles + (NEED_CAST_TILE ? 2u * STAGE_BYTES : 0u));
+    unsigned char *cast_tiles = io + (size_t)io_slots * io_arrays * F32_TILE_BYTES;
+    BulkShared *sh = reinterpret_cast<BulkShared *>(
+        cast_tiles + (NEED_CAST_TILE ? (size_t)io_slots * STAGE_BYTES : (size_t)0));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -495,7 +497,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
             ptx::mbar_init(&sh->sched_full[d], 1);
             ptx::mbar_init(&sh->sched_empty[d], BULK_ITEM_READERS);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < io_slots; ++b) {
             ptx::mbar_init(&sh->io_full[b], 1);
             ptx::mbar_init(&sh->io_empty[b], 1);
             ptx::mbar_init(&sh->out_ready[b], BULK_COMPUTE_WARPS);
@@ -517,7 +519,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
     long long k0;
     unsigned n;      // elements of the current tile (partial tiles: compute runs on the whole
                      // shared-memory tile, only the first n elements are loaded and stored)
-    unsigned t = 0;  // tiles seen by this role
+    RingPos io_pos;  // theta/momentum/result buffer of the current tile (advances once per tile)
     RingPos q;       // ring position of this role
 
     if (warp == BULK_COMPUTE_WARPS + 2) {
@@ -564,9 +566,9 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
         bool ok = true;
         while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
-            const int b = t & 1;
+            const int b = io_pos.slot;
             if (lane == 0) {
-                ok = bounded_wait(&sh->io_empty[b], ((t >> 1) & 1) ^ 1, p.error_word, 1);
+                ok = bounded_wait(&sh->io_empty[b], io_pos.phase ^ 1u, p.error_word, 1);
                 if (ok) {
                     const unsigned f32_bytes = n * 4u;
                     unsigned bytes = f32_bytes;
@@ -609,7 +611,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                 __syncwarp();
                 ok = __shfl_sync(0xffffffffu, ok, 0);
             }
-            ++t;
+            io_pos.advance(io_slots);
         }
         // Leave only when every copy this warp started has landed: another CTA may get this
         // shared memory next.  Waits on already completed phases return at once.
@@ -618,9 +620,9 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
                 q.retreat(stages);
                 bounded_wait(&sh->full[q.slot], q.phase, p.error_word, 3);
             }
-            for (unsigned back = 0; back < 2 && back < t; ++back) {
-                const unsigned tt = t - 1 - back;
-                bounded_wait(&sh->io_full[tt & 1], (tt >> 1) & 1, p.error_word, 3);
+            for (int back = 0; back < io_slots && io_pos.used > 0; ++back) {
+                io_pos.retreat(io_slots);
+                bounded_wait(&sh->io_full[io_pos.slot], io_pos.phase, p.error_word, 3);
             }
         }
     } else if (warp == BULK_COMPUTE_WARPS + 1) {
@@ -628,8 +630,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
         bool ok = true;
         while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
-            const int b = t & 1;
-            ok = bounded_wait(&sh->out_ready[b], (t >> 1) & 1, p.error_word, 4);
+            const int b = io_pos.slot;
+            ok = bounded_wait(&sh->out_ready[b], io_pos.phase, p.error_word, 4);
             if (!ok) break;
             if (lane == 0) {
                 if (pass.flags & KPASS_UPDATE) {
@@ -648,7 +650,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
             ptx::bulk_wait_read_all();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sh->io_empty[b]);
-            ++t;
+            io_pos.advance(io_slots);
         }
         ptx::bulk_wait_all();
     } else {
@@ -657,8 +659,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
         bool ok = true;
         while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
-            const int b = t & 1;
-            ok = bounded_wait(&sh->io_full[b], (t >> 1) & 1, p.error_word, 5);
+            const int b = io_pos.slot;
+            ok = bounded_wait(&sh->io_full[b], io_pos.phase, p.error_word, 5);
             if (!ok) break;
             float th[EPT], acc[EPT];
             float *th_tile = io_tile(b, 0);
@@ -755,7 +757,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays)
             ptx::fence_proxy_async();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sh->out_ready[b]);
-            ++t;
+            io_pos.advance(io_slots);
         }
     }
 }

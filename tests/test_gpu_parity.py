@@ -147,7 +147,8 @@ def test_kernel_families_and_tunings_agree_bitwise(dtype):
     for kernel, tuning in [(B.DIPACO_KERNEL_VECTOR, None), (B.DIPACO_KERNEL_AUTO, None),
                            (B.DIPACO_KERNEL_AUTO, (1, 3, 1)), (B.DIPACO_KERNEL_AUTO, (1, 0, 2)),
                            (B.DIPACO_KERNEL_AUTO, (2, 2, 1)), (B.DIPACO_KERNEL_AUTO, (1, 0, 4)),
-                           (B.DIPACO_KERNEL_AUTO, (3, 0, 1))]:
+                           (B.DIPACO_KERNEL_AUTO, (3, 0, 1)), (B.DIPACO_KERNEL_AUTO, (1, 6, 2, 4)),
+                           (B.DIPACO_KERNEL_AUTO, (1, 4, 1, 2))]:
         state = clone_problem(pr)
         run_gpu(pr, state, kernel=kernel, tuning=tuning)
         assert_states_bitwise_equal(ref, state)
