@@ -383,3 +383,50 @@ def test_gradient_rescaling_and_levels_kept_local(mode):
         assert_bf16_close(got[:n0], want_ps[i][:n0])
         assert_bf16_close(got[n0 + n1:], want_ps[i][n0 + n1:])
     assert not np.array_equal(got_th[:n0], before[0][:n0])
+
+
+def custom_problem(K, numel, table, dtype, seed, device=DEV, momentum_std=1e-4):
+    """A problem on an arbitrary path table (not the full product of the levels)."""
+    cfg = synth.SyncConfig("custom", tuple(K), tuple(numel), dtype, momentum_std=momentum_std, seed=seed)
+    table = np.ascontiguousarray(table, dtype=np.int32)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    theta = torch.empty(cfg.module_params, device=device).normal_(0, 0.02, generator=gen)
+    momentum = torch.empty(cfg.module_params, device=device).normal_(0, momentum_std, generator=gen)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    mod_off = np.concatenate([[0], np.cumsum([k * n for k, n in zip(K, numel)])])
+    paths = []
+    for i in range(table.shape[0]):
+        parts = []
+        for l, n in enumerate(numel):
+            src = int(mod_off[l]) + int(table[i, l]) * n
+            parts.append(theta[src:src + n] + torch.empty(n, device=device).normal_(0, 1e-3, generator=gen))
+        paths.append(torch.cat(parts).to(tdt))
+    return synth.SyncProblem(cfg, table, None, None, theta, momentum, paths)
+
+
+@pytest.mark.parametrize("case", ["diloco", "flat", "sampled_paths", "empty_level", "tiny_modules",
+                                  "many_paths"])
+def test_special_structures_match_the_oracle(case):
+    if case == "diloco":            # one level, one module, eight workers (Section 2.5)
+        pr = custom_problem((1,), (3 * 4096 + 40,), np.zeros((8, 1)), "bf16", 1)
+    elif case == "flat":            # no sharing at all: one level, K = P (Section 2.6.3)
+        pr = custom_problem((64,), (4096 + 24,), np.arange(64).reshape(64, 1), "bf16", 2)
+    elif case == "sampled_paths":   # three of the nine paths of a 3x3 grid; one module unused
+        pr = custom_problem((1, 3, 3), (4104, 2056, 4096), [[0, 0, 1], [0, 2, 1], [0, 2, 2]], "f32", 3)
+    elif case == "empty_level":     # a level without parameters
+        pr = custom_problem((1, 2, 2), (4096, 0, 2048 + 8), synth.path_table((1, 2, 2)), "bf16", 4)
+    elif case == "tiny_modules":    # modules smaller than one 16-byte unit
+        pr = custom_problem((1, 2, 2), (3, 1, 5), synth.path_table((1, 2, 2)), "bf16", 5)
+    else:                           # 1000 paths through one module, 125 modules of 8 paths
+        table = np.stack([np.zeros(1000, np.int64), np.arange(1000) // 8], axis=1)
+        pr = custom_problem((1, 125), (2 * 4096 + 16, 4096), table, "bf16", 6)
+    for chunk in (0, 3):
+        before = host_state(clone_problem(pr))
+        state = clone_problem(pr)
+        run_gpu(pr, state, chunk_paths=chunk)
+        assert_matches_oracle(pr, before, state)
+        if case == "sampled_paths":   # the module nobody passes through is never touched
+            n0, n1 = pr.cfg.level_numel[0], pr.cfg.level_numel[1]
+            sl = slice(n0 + n1, n0 + 2 * n1)
+            assert torch.equal(state[0][sl], pr.theta[sl]) and torch.equal(state[1][sl], pr.momentum[sl])
