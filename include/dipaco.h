@@ -152,6 +152,18 @@ int dipaco_set_module_scale(dipaco_ctx *ctx, const float *module_scale);
  */
 int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync);
 
+/*
+ * Sharded executor (Section 3.3, "Sharded Outer Optimization Executor": modules, and the
+ * parameters inside a module, are independent, so the update can be split over executors with no
+ * exchange between them).  This context then owns slab shard_index of shard_count of EVERY
+ * module (equal element ranges cut at multiples of 8192 elements; the last shard takes the
+ * remainder) and touches nothing else: theta, momentum and the path copies outside its slabs are
+ * neither read nor written.  Pointers and layouts stay those of the whole problem, so S contexts
+ * (one per GPU, each holding at least its slabs at the usual offsets) together perform exactly
+ * the unsharded update, bit for bit.  Default: shard 0 of 1.
+ */
+int dipaco_set_shard(dipaco_ctx *ctx, int32_t shard_index, int32_t shard_count);
+
 /* Choose the kernel family (DIPACO_KERNEL_*); all families give bitwise identical results. */
 int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
 

@@ -40,7 +40,7 @@ EXPORTS = [
     "dipaco_device_status", "dipaco_launch_count", "dipaco_plan_module", "dipaco_plan_offsets",
     "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
     "dipaco_set_host_unit_bytes", "dipaco_plan_traffic", "dipaco_set_module_scale",
-    "dipaco_set_level_sync",
+    "dipaco_set_level_sync", "dipaco_set_shard",
 ]
 
 _lib = None
@@ -76,6 +76,7 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_weights.argtypes = [vp, vp]
     lib.dipaco_set_module_scale.argtypes = [vp, vp]
     lib.dipaco_set_level_sync.argtypes = [vp, vp]
+    lib.dipaco_set_shard.argtypes = [vp, i32, i32]
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32, i32]
     lib.dipaco_device_status.argtypes = [vp]
@@ -201,6 +202,10 @@ def dipaco_set_module_scale(ctx, module_scale) -> None:
 def dipaco_set_level_sync(ctx, level_sync) -> None:
     ls = None if level_sync is None else np.ascontiguousarray(level_sync, dtype=np.uint8)
     _check(load().dipaco_set_level_sync(ctx, _np_ptr(ls)), "dipaco_set_level_sync")
+
+
+def dipaco_set_shard(ctx, shard_index: int, shard_count: int) -> None:
+    _check(load().dipaco_set_shard(ctx, int(shard_index), int(shard_count)), "dipaco_set_shard")
 
 
 def dipaco_set_kernel(ctx, kernel: int) -> None:

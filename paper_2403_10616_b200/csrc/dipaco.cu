@@ -585,6 +585,15 @@ int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync)
     return DIPACO_OK;
 }
 
+int dipaco_set_shard(dipaco_ctx *ctx, int32_t shard_index, int32_t shard_count)
+{
+    if (!ctx || shard_count < 1 || shard_index < 0 || shard_index >= shard_count) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ctx->grid.shard_index = shard_index;
+    ctx->grid.shard_count = shard_count;
+    return DIPACO_OK;
+}
+
 int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel)
 {
     if (!ctx || kernel < DIPACO_KERNEL_AUTO || kernel > DIPACO_KERNEL_SCALAR) return DIPACO_EINVAL;
@@ -850,7 +859,8 @@ int dipaco_plan_traffic(const dipaco_ctx *ctx, const uint8_t *reported, int64_t 
             if (specs.empty()) return;
             ++count;
             for (const PassSpec &sp : specs)
-                total += pass_cost_per_elem(sp, ctx->elem_size) * (double)g.modules[sp.module].numel;
+                total += pass_cost_per_elem(sp, ctx->elem_size) *
+                         (double)((sp.end < 0 ? g.modules[sp.module].numel : sp.end) - sp.begin);
         };
         if (g.num_chunks <= 1) {
             plan_resident(g, mc, specs);

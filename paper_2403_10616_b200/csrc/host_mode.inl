@@ -134,8 +134,10 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
         if ((size_t)slab * es > h->stage_out_bytes)
             slab = (int64_t)(h->stage_out_bytes / (size_t)es) / tile * tile;
         if (slab < 1) return DIPACO_ENOMEM;
-        for (int64_t a = 0; a < m.numel; a += slab, ++unit_index) {
-            const int64_t b = std::min<int64_t>(m.numel, a + slab);
+        int64_t shard_lo = 0, shard_hi = m.numel;
+        g.shard_range(m, shard_lo, shard_hi);
+        for (int64_t a = shard_lo; a < shard_hi; a += slab, ++unit_index) {
+            const int64_t b = std::min<int64_t>(shard_hi, a + slab);
             const int buf = (int)(unit_index & 1);
             const size_t piece = (size_t)(b - a) * es;
             const size_t piece_stride = align_up(piece, 256);

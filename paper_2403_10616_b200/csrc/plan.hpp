@@ -39,10 +39,25 @@ struct Grid {
     int64_t module_params = 0, params_per_path = 0;
     int chunk_paths = 0, num_chunks = 1;
     int64_t scratch_elems = 0;
+    int shard_index = 0, shard_count = 1;  // this context owns one slab of every module
 
     int module_id(int l, int e) const { return level_first[l] + e; }
     bool synced(const ModuleGeom &m) const { return level_sync.empty() || level_sync[(size_t)m.level]; }
     float scale_of(size_t id) const { return module_scale.empty() ? 1.0f : module_scale[id]; }
+    // Element range of a module that this shard owns: equal slabs cut at multiples of 8192
+    // elements (a multiple of every tile size), the last shard takes the remainder.
+    void shard_range(const ModuleGeom &m, int64_t &lo, int64_t &hi) const
+    {
+        const int64_t grain = 8192;
+        auto cut = [&](int i) -> int64_t {
+            if (i <= 0) return 0;
+            if (i >= shard_count) return m.numel;
+            const int64_t c = (int64_t)((__int128)m.numel * i / shard_count);
+            return c / grain * grain;
+        };
+        lo = cut(shard_index);
+        hi = cut(shard_index + 1);
+    }
     int chunk_of(int path) const { return chunk_paths > 0 ? path / chunk_paths : 0; }
 };
 
@@ -155,6 +170,8 @@ inline void plan_resident(const Grid &g, const std::vector<ModuleCoeffs> &mc,
         if (m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
         PassSpec p;
         p.module = (int)id;
+        g.shard_range(m, p.begin, p.end);
+        if (p.begin >= p.end) continue;
         p.scale = g.scale_of(id);
         p.flags = mc[id].update ? PASS_UPDATE : 0;
         p.contributors = mc[id].contributors;
@@ -177,6 +194,8 @@ inline void plan_accumulate(const Grid &g, const std::vector<ModuleCoeffs> &mc, 
         const int last = g.chunk_of(k.contributors.back());
         PassSpec p;
         p.module = (int)id;
+        g.shard_range(m, p.begin, p.end);
+        if (p.begin >= p.end) continue;
         p.scale = g.scale_of(id);
         for (size_t j = 0; j < k.contributors.size(); ++j)
             if (g.chunk_of(k.contributors[j]) == c) {
@@ -209,6 +228,8 @@ inline void plan_writeback(const Grid &g, const std::vector<ModuleCoeffs> &mc, i
         if (skip_final && k.update && g.chunk_of(k.contributors.back()) == c) continue;
         PassSpec p;
         p.module = (int)id;
+        g.shard_range(m, p.begin, p.end);
+        if (p.begin >= p.end) continue;
         p.flags = 0;
         for (int i : m.members)
             if (g.chunk_of(i) == c) p.members.push_back(i);

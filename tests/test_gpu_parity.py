@@ -430,3 +430,42 @@ def test_special_structures_match_the_oracle(case):
             n0, n1 = pr.cfg.level_numel[0], pr.cfg.level_numel[1]
             sl = slice(n0 + n1, n0 + 2 * n1)
             assert torch.equal(state[0][sl], pr.theta[sl]) and torch.equal(state[1][sl], pr.momentum[sl])
+
+
+@pytest.mark.parametrize("mode", ["resident", "chunked", "host"])
+def test_shards_together_equal_the_unsharded_update(mode):
+    """Three contexts, each owning one slab of every module, applied one after another to the same
+    buffers, give bitwise the unsharded result; each touches only its own slabs."""
+    base = synth.CONFIGS["grid4x4"]
+    cfg = synth.SyncConfig("shards", (1, 4, 4), (5 * 8192 + 4096 + 24, 3 * 8192 + 8, 2 * 8192 + 1003),
+                           "bf16", weights="tokens", momentum_std=1e-4, mask_prob=0.2, seed=11)
+    dev = "cpu" if mode == "host" else DEV
+    pr = synth.make_problem(cfg, dev)
+    whole = clone_problem(pr)
+    ctx = make_ctx(pr, chunk_paths=0 if mode == "resident" else 5)
+
+    def call(state):
+        ptrs = [p.data_ptr() for p in state[2]]
+        fn = B.dipaco_outer_sync_host if mode == "host" else B.dipaco_outer_sync
+        fn(ctx, state[0].data_ptr(), state[1].data_ptr(), ptrs, pr.reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+
+    call(whole)
+    parts = clone_problem(pr)
+    changed_so_far = torch.zeros_like(parts[0], dtype=torch.bool)
+    for shard in range(3):
+        B.dipaco_set_shard(ctx, shard, 3)
+        before = parts[0].clone()
+        call(parts)
+        changed = parts[0] != before
+        assert changed.any() and not (changed & changed_so_far).any()
+        changed_so_far |= changed
+    B.dipaco_set_shard(ctx, 0, 1)
+    B.dipaco_destroy(ctx)
+    assert_states_bitwise_equal(whole, parts)
+    with pytest.raises(B.DipacoError):
+        c2 = make_ctx(pr)
+        try:
+            B.dipaco_set_shard(c2, 3, 3)
+        finally:
+            B.dipaco_destroy(c2)

@@ -230,3 +230,19 @@ def test_planned_traffic_of_resident_mode_is_the_algorithmic_minimum():
     nbytes, launches = B.dipaco_plan_traffic(ctx)
     assert launches == 15 and 1.4 < nbytes / synth.algorithmic_bytes(cfg) < 1.6
     B.dipaco_destroy(ctx)
+
+
+def test_shards_partition_the_planned_traffic():
+    cfg = synth.CONFIGS["grid16x16"]
+    ctx = plan_ctx(cfg)
+    whole, _ = B.dipaco_plan_traffic(ctx)
+    parts = []
+    for shard in range(8):
+        B.dipaco_set_shard(ctx, shard, 8)
+        parts.append(B.dipaco_plan_traffic(ctx)[0])
+    assert sum(parts) == whole
+    assert max(parts) - min(parts) < 0.001 * whole     # equal slabs up to the 8192-element grain
+    for bad in ((8, 8), (-1, 8), (0, 0)):
+        with pytest.raises(B.DipacoError):
+            B.dipaco_set_shard(ctx, *bad)
+    B.dipaco_destroy(ctx)
