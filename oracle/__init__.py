@@ -22,6 +22,10 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 F32 = 0
 BF16 = 1
 
+NESTEROV = 0
+MOMENTUM = 1
+SGD = 2
+
 _lib = None
 
 
@@ -49,8 +53,8 @@ def _load():
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
         ]
         lib.oracle_outer_sync_ex.restype = ctypes.c_int
-        lib.oracle_outer_sync_ex.argtypes = lib.oracle_outer_sync.argtypes + [ctypes.c_void_p,
-                                                                              ctypes.c_void_p]
+        lib.oracle_outer_sync_ex.argtypes = lib.oracle_outer_sync.argtypes + [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32]
         lib.oracle_max_threads.restype = ctypes.c_int32
         lib.oracle_max_threads.argtypes = []
         _lib = lib
@@ -63,7 +67,7 @@ def max_threads() -> int:
 
 def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, paths,
                path_dtype, outer_lr, outer_momentum, path_weights=None, reported=None,
-               num_threads=1, module_scale=None, level_sync=None):
+               num_threads=1, module_scale=None, level_sync=None, optimizer=NESTEROV):
     """Run one outer synchronisation in place on host arrays.
 
     theta, momentum: contiguous float32 numpy arrays of sum_l K_l*N_l elements (level, module,
@@ -72,6 +76,7 @@ def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, 
     path_weights: None (uniform) or [P] float32.  reported: None (all) or [P] of 0/1.
     module_scale: None or [sum_l K_l] factors on the modules' outer gradients (level-major).
     level_sync: None or [L] of 0/1, 0 = the level is left untouched.
+    optimizer: NESTEROV (the paper's), MOMENTUM (heavy ball) or SGD.
     """
     lib = _load()
     K = np.ascontiguousarray(modules_per_level, dtype=np.int32)
@@ -114,6 +119,7 @@ def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, 
         int(num_threads),
         sc.ctypes.data if sc is not None else None,
         ls.ctypes.data if ls is not None else None,
+        int(optimizer),
     )
     if rc != 0:
         raise ValueError("oracle_outer_sync rejected its arguments")

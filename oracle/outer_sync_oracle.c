@@ -33,6 +33,12 @@
  *     blocks of the path-specific models local to their path): theta, momentum and every copy
  *     of its modules are left untouched.
  *
+ *   - optimizer: Section 2.5 notes that other outer optimisers of the federated family fit the
+ *     same scheme.  Besides Nesterov (0, the paper's choice) the oracle defines heavy-ball
+ *     momentum (1): m' = mu*m + Delta, theta' = theta - lr*m'; and plain SGD (2):
+ *     theta' = theta - lr*Delta with the momentum buffer left as it is (lr = 1 is plain
+ *     averaging of the copies).
+ *
  * Arithmetic: steps 1-3 in double, theta' and m' rounded once to float;
  * a bf16 path copy receives round-to-nearest-even of that float.
  * Loop order: module, element, contributor (ascending path id).
@@ -109,6 +115,7 @@ static void write_copy(void *buf, int dtype, int64_t idx, float v)
  *
  *  module_scale        [sum_l K_l] factor on each module's outer gradient, level-major, or NULL = 1
  *  level_sync          [L] 0 = leave the level untouched, or NULL = every level is synchronised
+ *  optimizer           0 = Nesterov momentum, 1 = heavy-ball momentum, 2 = plain SGD
  *
  * Returns 0, or -1 on an invalid argument.
  */
@@ -118,8 +125,10 @@ int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
                          const uint8_t *reported, double outer_lr, double outer_momentum,
                          int32_t path_dtype, float *theta, float *momentum,
                          void *const *path_ptrs, int32_t num_threads,
-                         const double *module_scale, const uint8_t *level_sync)
+                         const double *module_scale, const uint8_t *level_sync, int32_t optimizer)
 {
+    if (optimizer < 0 || optimizer > 2)
+        return -1;
     if (num_levels < 1 || num_paths < 1 || !modules_per_level || !level_numel ||
         !path_to_module || !theta || !momentum || !path_ptrs)
         return -1;
@@ -190,8 +199,17 @@ int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
                         delta += alpha[r] * (t0 - x);
                     }
                     delta *= scale;
-                    const double m1 = outer_momentum * (double)mo[k] + delta;
-                    const double t1 = t0 - outer_lr * (delta + outer_momentum * m1);
+                    double m1, t1;
+                    if (optimizer == 0) {          /* Nesterov momentum */
+                        m1 = outer_momentum * (double)mo[k] + delta;
+                        t1 = t0 - outer_lr * (delta + outer_momentum * m1);
+                    } else if (optimizer == 1) {   /* heavy-ball momentum */
+                        m1 = outer_momentum * (double)mo[k] + delta;
+                        t1 = t0 - outer_lr * m1;
+                    } else {                       /* plain SGD, momentum buffer untouched */
+                        m1 = (double)mo[k];
+                        t1 = t0 - outer_lr * delta;
+                    }
                     mo[k] = (float)m1;
                     new_theta = (float)t1;
                     th[k] = new_theta;
@@ -216,7 +234,7 @@ int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
 {
     return oracle_outer_sync_ex(num_levels, modules_per_level, level_numel, num_paths,
                                 path_to_module, path_weights, reported, outer_lr, outer_momentum,
-                                path_dtype, theta, momentum, path_ptrs, num_threads, NULL, NULL);
+                                path_dtype, theta, momentum, path_ptrs, num_threads, NULL, NULL, 0);
 }
 
 /* number of OpenMP threads the element loop can use on this host (1 without OpenMP) */

@@ -32,7 +32,8 @@ def host_copy(problem):
 
 
 def run_oracle(cfg, table, theta, momentum, paths, weights=None, reported=None,
-               lr=None, mu=None, num_threads=1, module_scale=None, level_sync=None):
+               lr=None, mu=None, num_threads=1, module_scale=None, level_sync=None,
+               optimizer=0):
     """Oracle on copies of the given host arrays; returns (theta', m', [copies'])."""
     th = theta.copy()
     mo = momentum.copy()
@@ -41,7 +42,8 @@ def run_oracle(cfg, table, theta, momentum, paths, weights=None, reported=None,
     lr = np.float32(cfg.outer_lr if lr is None else lr)
     mu = np.float32(cfg.outer_momentum if mu is None else mu)
     oracle.outer_sync(cfg.modules_per_level, cfg.level_numel, table, th, mo, ps, dtype,
-                      float(lr), float(mu), weights, reported, num_threads, module_scale, level_sync)
+                      float(lr), float(mu), weights, reported, num_threads, module_scale, level_sync,
+                      optimizer)
     return th, mo, ps
 
 

@@ -486,3 +486,52 @@ def test_levels_flagged_as_not_communicated_are_left_untouched():
     np.testing.assert_array_equal(got_th[:6], full_th[:6])
     np.testing.assert_array_equal(got_th[16:], full_th[16:])
     np.testing.assert_array_equal(got_mo[16:], full_mo[16:])
+
+
+# ---------------------------------------------------------------------------- other outer optimisers
+
+@pytest.mark.parametrize("kind,nesterov", [(oracle.MOMENTUM, False), (oracle.NESTEROV, True)])
+def test_momentum_variants_match_the_library_sgd(kind, nesterov):
+    """Three rounds against torch.optim.SGD(momentum, nesterov=...) fed with numpy's mean."""
+    cfg = synth.SyncConfig("dense", (1,), (129,), "f32")
+    table = np.zeros((4, 1), dtype=np.int32)
+    rng = np.random.RandomState(4)
+    theta = rng.normal(0, 0.02, 129).astype(np.float32)
+    momentum = np.zeros(129, dtype=np.float32)
+    param = torch.nn.Parameter(torch.from_numpy(theta.copy()).double())
+    opt = torch.optim.SGD([param], lr=LR, momentum=MU, nesterov=nesterov)
+    for rnd in range(3):
+        paths = [(theta + rng.normal(0, 1e-3, 129)).astype(np.float32) for _ in range(4)]
+        delta = np.mean(np.stack([theta.astype(np.float64) - p.astype(np.float64) for p in paths]), axis=0)
+        with torch.no_grad():
+            param.copy_(torch.from_numpy(theta.astype(np.float64)))
+        if rnd > 0:   # the oracle keeps its momentum in fp32: start the library step from the same state
+            opt.state[param]["momentum_buffer"] = torch.from_numpy(momentum.astype(np.float64))
+        param.grad = torch.from_numpy(delta.copy())
+        opt.step()
+        theta, momentum, _ = helpers.run_oracle(cfg, table, theta, momentum, paths, optimizer=kind)
+        want = param.detach().numpy()
+        assert np.all(np.abs(theta - want) <= one_ulp(want))
+
+
+def test_heavy_ball_constant_gradient_series_and_plain_sgd():
+    cfg = tiny_cfg((1,), (2,))
+    table = synth.path_table(cfg.modules_per_level)
+    theta = np.array([4.0, -1.0], dtype=np.float32)
+    momentum = np.zeros(2, dtype=np.float32)
+    # heavy ball under g = 1: m_T = (1 - mu^T)/(1 - mu), step_T = lr * m_T  -> 0.7, 1.33, 1.897
+    for want_step in (0.7, 1.33, 1.897):
+        new_th, momentum, _ = helpers.run_oracle(cfg, table, theta, momentum, [theta - np.float32(1.0)],
+                                                 optimizer=oracle.MOMENTUM)
+        np.testing.assert_allclose(theta - new_th, want_step, rtol=0, atol=4e-6)
+        theta = new_th
+    # plain SGD with lr = 1 is the mean of the copies and leaves the momentum buffer alone
+    cfg = tiny_cfg((1, 2), (5, 4), momentum_std=1e-2, seed=31)
+    pr = synth.make_problem(cfg)
+    th, mo, ps = helpers.host_copy(pr)
+    got_th, got_mo, _ = helpers.run_oracle(cfg, pr.table, th, mo, ps, lr=1.0, optimizer=oracle.SGD)
+    np.testing.assert_array_equal(got_mo, mo)
+    want = np.mean(np.stack([p[:5].astype(np.float64) for p in ps]), axis=0)
+    assert np.all(np.abs(got_th[:5] - want) <= one_ulp(want))
+    with pytest.raises(ValueError):
+        helpers.run_oracle(cfg, pr.table, th, mo, ps, optimizer=3)
