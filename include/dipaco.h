@@ -55,6 +55,13 @@ enum {
     DIPACO_ELIMIT = -7    /* a size exceeds a fixed limit of the entry point (static scratch)   */
 };
 
+/* outer optimisers for dipaco_set_optimizer */
+enum {
+    DIPACO_OPT_NESTEROV = 0, /* m' = mu*m + Delta; theta' = theta - lr*(Delta + mu*m')   (the paper's) */
+    DIPACO_OPT_MOMENTUM = 1, /* m' = mu*m + Delta; theta' = theta - lr*m'                (heavy ball)  */
+    DIPACO_OPT_SGD = 2       /* theta' = theta - lr*Delta; momentum left as it is (lr = 1: averaging)   */
+};
+
 /* kernel selection for dipaco_set_kernel */
 enum {
     DIPACO_KERNEL_AUTO = 0,   /* bulk-copy (TMA) pipeline for 16-byte aligned full tiles, scalar rest */
@@ -151,6 +158,12 @@ int dipaco_set_module_scale(dipaco_ctx *ctx, const float *module_scale);
  * of the level's modules are left untouched; NULL = every level is synchronised.
  */
 int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync);
+
+/*
+ * Outer optimiser (Section 2.5: Nesterov momentum is the paper's choice; other optimisers of the
+ * federated family fit the same scheme).  DIPACO_OPT_*; the default is Nesterov.
+ */
+int dipaco_set_optimizer(dipaco_ctx *ctx, int32_t optimizer);
 
 /*
  * Sharded executor (Section 3.3, "Sharded Outer Optimization Executor": modules, and the

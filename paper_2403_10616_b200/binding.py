@@ -29,6 +29,10 @@ DIPACO_ENODEV = -6
 DIPACO_ELIMIT = -7
 DIPACO_STATIC_MAX_NUMEL = 4 * 1024 * 1024
 
+DIPACO_OPT_NESTEROV = 0
+DIPACO_OPT_MOMENTUM = 1
+DIPACO_OPT_SGD = 2
+
 DIPACO_KERNEL_AUTO = 0
 DIPACO_KERNEL_VECTOR = 1
 DIPACO_KERNEL_SCALAR = 2
@@ -40,7 +44,7 @@ EXPORTS = [
     "dipaco_device_status", "dipaco_launch_count", "dipaco_plan_module", "dipaco_plan_offsets",
     "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
     "dipaco_set_host_unit_bytes", "dipaco_plan_traffic", "dipaco_set_module_scale",
-    "dipaco_set_level_sync", "dipaco_set_shard",
+    "dipaco_set_level_sync", "dipaco_set_shard", "dipaco_set_optimizer",
 ]
 
 _lib = None
@@ -77,6 +81,7 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_module_scale.argtypes = [vp, vp]
     lib.dipaco_set_level_sync.argtypes = [vp, vp]
     lib.dipaco_set_shard.argtypes = [vp, i32, i32]
+    lib.dipaco_set_optimizer.argtypes = [vp, i32]
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32, i32]
     lib.dipaco_device_status.argtypes = [vp]
@@ -202,6 +207,10 @@ def dipaco_set_module_scale(ctx, module_scale) -> None:
 def dipaco_set_level_sync(ctx, level_sync) -> None:
     ls = None if level_sync is None else np.ascontiguousarray(level_sync, dtype=np.uint8)
     _check(load().dipaco_set_level_sync(ctx, _np_ptr(ls)), "dipaco_set_level_sync")
+
+
+def dipaco_set_optimizer(ctx, optimizer: int) -> None:
+    _check(load().dipaco_set_optimizer(ctx, int(optimizer)), "dipaco_set_optimizer")
 
 
 def dipaco_set_shard(ctx, shard_index: int, shard_count: int) -> None:

@@ -49,6 +49,7 @@ struct HostMode;  // state of dipaco_outer_sync_host (host_mode.inl)
 struct dipaco_ctx {
     Grid grid;
     float lr = 0.f, mu = 0.f;
+    int optimizer = DIPACO_OPT_NESTEROV;
     int dtype = DIPACO_F32;
     int elem_size = 4;
     int device = -1;
@@ -383,6 +384,7 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
     lp.members = reinterpret_cast<void *const *>(base + pl.members_off);
     lp.lr = ctx->lr;
     lp.mu = ctx->mu;
+    lp.optimizer = ctx->optimizer;
     lp.error_word = ctx->error_word;
     lp.num_passes = pl.num_passes;
     lp.total_items = pl.total_items;
@@ -582,6 +584,14 @@ int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync)
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
     if (level_sync) ctx->grid.level_sync.assign(level_sync, level_sync + ctx->grid.L);
     else ctx->grid.level_sync.clear();
+    return DIPACO_OK;
+}
+
+int dipaco_set_optimizer(dipaco_ctx *ctx, int32_t optimizer)
+{
+    if (!ctx || optimizer < DIPACO_OPT_NESTEROV || optimizer > DIPACO_OPT_SGD) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ctx->optimizer = optimizer;
     return DIPACO_OK;
 }
 

@@ -56,6 +56,7 @@ struct LaunchParams {
     const SegmentDev *segs;
     const int *cta_first;  // [gridDim.x + 1]
     float lr, mu;
+    int optimizer;  // KOPT_*
     int *error_word;
     // bulk-copy kernel only
     int num_passes;
@@ -65,7 +66,7 @@ struct LaunchParams {
 };
 
 // ------------------------------------------------------------------------------------------
-// The arithmetic, written once.  Explicit intrinsics: no contraction or reassociation choices
+// The arithmetic, written once (sync_accumulate, sync_update).  Explicit intrinsics: no contraction or reassociation choices
 // are left to the compiler, so every kernel family rounds identically.
 
 __device__ __forceinline__ float sync_accumulate(float acc, float c, float theta, float x)
@@ -74,13 +75,23 @@ __device__ __forceinline__ float sync_accumulate(float acc, float c, float theta
     return __fmaf_rn(c, __fsub_rn(theta, x), acc);
 }
 
-__device__ __forceinline__ void sync_nesterov(float theta, float m, float sum, float scale, float lr,
-                                              float mu, float &theta_new, float &m_new)
+enum : int { KOPT_NESTEROV = 0, KOPT_MOMENTUM = 1, KOPT_SGD = 2 };
+
+__device__ __forceinline__ void sync_update(float theta, float m, float sum, float scale, float lr,
+                                            float mu, int optimizer, float &theta_new, float &m_new)
 {
-    // Delta = scale * sum ; m' = mu*m + Delta ; theta' = theta - lr*(Delta + mu*m')
+    // Delta = scale * sum, then the outer optimiser step:
+    //   Nesterov   m' = mu*m + Delta ; theta' = theta - lr*(Delta + mu*m')
+    //   heavy ball m' = mu*m + Delta ; theta' = theta - lr*m'
+    //   SGD        m' = m            ; theta' = theta - lr*Delta
     const float delta = __fmul_rn(scale, sum);  // exact when scale == 1
+    if (optimizer == KOPT_SGD) {
+        m_new = m;
+        theta_new = __fmaf_rn(-lr, delta, theta);
+        return;
+    }
     m_new = __fmaf_rn(mu, m, delta);
-    const float g = __fmaf_rn(mu, m_new, delta);
+    const float g = optimizer == KOPT_NESTEROV ? __fmaf_rn(mu, m_new, delta) : m_new;
     theta_new = __fmaf_rn(-lr, g, theta);
 }
 
@@ -256,7 +267,7 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
 #pragma unroll
                 for (int v = 0; v < VEC; ++v) {
                     float t1, m1;
-                    sync_nesterov(th[v], mo[v], acc[v], pass.scale, p.lr, p.mu, t1, m1);
+                    sync_update(th[v], mo[v], acc[v], pass.scale, p.lr, p.mu, p.optimizer, t1, m1);
                     th[v] = t1;
                     mo[v] = m1;
                 }
@@ -738,8 +749,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                         float m1[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            sync_nesterov(th[u * UE + v + i], mo[i], acc[u * UE + v + i], pass.scale, p.lr,
-                                          p.mu, th[u * UE + v + i], m1[i]);
+                            sync_update(th[u * UE + v + i], mo[i], acc[u * UE + v + i], pass.scale, p.lr,
+                                        p.mu, p.optimizer, th[u * UE + v + i], m1[i]);
                         *reinterpret_cast<float4 *>(mo_tile + e0 + v) =
                             make_float4(m1[0], m1[1], m1[2], m1[3]);
                         *reinterpret_cast<float4 *>(th_tile + e0 + v) =

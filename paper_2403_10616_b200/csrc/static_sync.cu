@@ -37,7 +37,7 @@ struct StaticWritebackArgs {
     int count;
 };
 
-// One element per thread, any alignment; the same arithmetic (sync_accumulate, sync_nesterov) and
+// One element per thread, any alignment; the same arithmetic (sync_accumulate, sync_update) and
 // the same order as the context-based kernels.
 template <typename PathT>
 __global__ void __launch_bounds__(256) static_accumulate_kernel(StaticAccumulateArgs a)
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(256) static_accumulate_kernel(StaticAccumulate
         if (a.flags & KPASS_PARTIAL_OUT) a.partial[k] = acc;
         if (a.flags & KPASS_UPDATE) {
             float t1, m1;
-            sync_nesterov(th, a.momentum[k], acc, 1.0f, a.lr, a.mu, t1, m1);
+            sync_update(th, a.momentum[k], acc, 1.0f, a.lr, a.mu, KOPT_NESTEROV, t1, m1);
             a.theta[k] = t1;
             a.momentum[k] = m1;
         }

@@ -469,3 +469,33 @@ def test_shards_together_equal_the_unsharded_update(mode):
             B.dipaco_set_shard(c2, 3, 3)
         finally:
             B.dipaco_destroy(c2)
+
+
+@pytest.mark.parametrize("opt", [B.DIPACO_OPT_MOMENTUM, B.DIPACO_OPT_SGD])
+@pytest.mark.parametrize("chunk", [0, 32])
+def test_other_outer_optimizers_match_the_oracle(opt, chunk):
+    base = synth.CONFIGS["grid16x16-masked"]
+    cfg = dataclass_replace(base.scaled((4096 + 72, 4096 + 8, 2 * 4096 + 1003)), momentum_std=1e-4)
+    pr = synth.make_problem(cfg, DEV)
+    before = host_state(clone_problem(pr))
+    theta, momentum, paths = clone_problem(pr)
+    ctx = make_ctx(pr, chunk_paths=chunk)
+    B.dipaco_set_optimizer(ctx, opt)
+    B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths],
+                        pr.reported)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    B.dipaco_destroy(ctx)
+    want_th, want_mo, want_ps = helpers.run_oracle(cfg, pr.table, *before, pr.weights, pr.reported,
+                                                   num_threads=8, optimizer=int(opt))
+    for got, want in ((helpers.tensor_to_numpy(theta), want_th), (helpers.tensor_to_numpy(momentum), want_mo)):
+        err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+        assert np.all(err <= 1e-6 * (1.0 + np.abs(want.astype(np.float64))))
+    if opt == B.DIPACO_OPT_SGD:
+        assert torch.equal(momentum.view(torch.int32), pr.momentum.view(torch.int32))
+    for i in range(0, cfg.num_paths, 7):
+        assert_bf16_close(helpers.tensor_to_numpy(paths[i]), want_ps[i])
+
+
+def dataclass_replace(cfg, **kw):
+    import dataclasses
+    return dataclasses.replace(cfg, **kw)
