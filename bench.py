@@ -37,7 +37,7 @@ REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the referen
 # figure is this ratio times the algorithmic bytes.  Only valid for the kernel source it was taken
 # from: the digest below is checked and "traffic" is null after any change to the kernels.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9918
-NCU_CAPTURE_KERNELS_SHA256 = "98d96b4add4d32686e689781009bc1b4ccf6022105b8f0003f5f5bf966e0cd8d"
+NCU_CAPTURE_KERNELS_SHA256 = "6f065115d04dc84075abaf1f7c5476aabe790afffa45717ae59d748ac4f9d66f"
 
 
 def kernels_digest():
