@@ -2,9 +2,7 @@
 // Host side: argument checks, planning (plan.hpp), table upload, kernel launches (kernels.cuh).
 #include "../../include/dipaco.h"
 
-#include <cstdio>
 #include <cstring>
-#include <functional>
 #include <new>
 #include <vector>
 
@@ -75,10 +73,8 @@ struct dipaco_ctx {
     float *theta = nullptr, *momentum = nullptr;
     cudaStream_t stream = nullptr;
     cudaStream_t last_stream = nullptr;
-    std::vector<uint8_t> mask;       // copy of `reported` (empty = all reported)
     std::vector<ModuleCoeffs> coeffs;
     int next_chunk = 0;
-    std::vector<uint8_t> written_back;
 
     HostMode *host_mode = nullptr;
 };
@@ -656,10 +652,7 @@ int dipaco_sync_begin(dipaco_ctx *ctx, float *theta, float *momentum, const uint
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
     if (ctx->grid.chunk_paths <= 0) return DIPACO_ESTATE;
     try {
-        if (reported) ctx->mask.assign(reported, reported + ctx->grid.P);
-        else ctx->mask.clear();
         compute_all_coeffs(ctx, reported);
-        ctx->written_back.assign((size_t)ctx->grid.num_chunks, 0);
     } catch (const std::bad_alloc &) {
         return DIPACO_ENOMEM;
     }
@@ -717,7 +710,6 @@ int dipaco_sync_writeback(dipaco_ctx *ctx, int32_t chunk_index, void *const *chu
     } catch (const std::bad_alloc &) {
         return DIPACO_ENOMEM;
     }
-    ctx->written_back[(size_t)chunk_index] = 1;
     return DIPACO_OK;
 }
 
