@@ -287,7 +287,9 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": cfg.name, "sample": sample},
+        "config": {"workload": cfg.name, "levels": list(cfg.modules_per_level),
+                   "level_numel": list(cfg.level_numel), "paths": cfg.num_paths,
+                   "path_dtype": cfg.path_dtype, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

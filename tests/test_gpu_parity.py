@@ -499,3 +499,34 @@ def test_other_outer_optimizers_match_the_oracle(opt, chunk):
 def dataclass_replace(cfg, **kw):
     import dataclasses
     return dataclasses.replace(cfg, **kw)
+
+
+def test_calls_run_on_the_callers_stream():
+    """Work is ordered on the stream that is passed in: producer and consumer kernels queued on a
+    side stream around the call see consistent data without any device-wide synchronisation."""
+    cfg = synth.CONFIGS["grid4x4"].scaled((6 * 4096 + 8, 4096 + 16, 2 * 4096))
+    pr = synth.make_problem(cfg, DEV)
+    ref = clone_problem(pr)
+    run_gpu(pr, ref)
+    side = torch.cuda.Stream()
+    theta, momentum, paths = clone_problem(pr)
+    torch.cuda.synchronize()
+    ctx = make_ctx(pr)
+    with torch.cuda.stream(side):
+        # inputs are produced on the side stream right before the call ...
+        staged = [p.clone() for p in paths]
+        for p in paths:
+            p.zero_()
+        for p, q in zip(paths, staged):
+            p.copy_(q)
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths],
+                            pr.reported, stream=side)
+        # ... and consumed on it right after
+        total = sum(float(p.double().sum()) for p in paths[:2])
+    side.synchronize()
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    B.dipaco_destroy(ctx)
+    want = sum(float(p.double().sum()) for p in ref[2][:2])
+    assert abs(total - want) <= 1e-4 * (1 + abs(want))
+    err = (theta.double() - ref[0].double()).abs()
+    assert bool((err <= 1e-6 * (1 + ref[0].double().abs())).all())
