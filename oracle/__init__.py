@@ -25,6 +25,10 @@ BF16 = 1
 NESTEROV = 0
 MOMENTUM = 1
 SGD = 2
+ADAM = 3
+
+COPIES = 0
+GRADIENTS = 1
 
 _lib = None
 
@@ -54,6 +58,7 @@ def _load():
         ]
         lib.oracle_outer_sync_ex.restype = ctypes.c_int
         lib.oracle_outer_sync_ex.argtypes = lib.oracle_outer_sync.argtypes + [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32]
         lib.oracle_max_threads.restype = ctypes.c_int32
         lib.oracle_max_threads.argtypes = []
@@ -67,7 +72,8 @@ def max_threads() -> int:
 
 def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, paths,
                path_dtype, outer_lr, outer_momentum, path_weights=None, reported=None,
-               num_threads=1, module_scale=None, level_sync=None, optimizer=NESTEROV):
+               num_threads=1, module_scale=None, level_sync=None, optimizer=NESTEROV,
+               second_moment=None, adam=None, input_kind=COPIES):
     """Run one outer synchronisation in place on host arrays.
 
     theta, momentum: contiguous float32 numpy arrays of sum_l K_l*N_l elements (level, module,
@@ -76,7 +82,9 @@ def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, 
     path_weights: None (uniform) or [P] float32.  reported: None (all) or [P] of 0/1.
     module_scale: None or [sum_l K_l] factors on the modules' outer gradients (level-major).
     level_sync: None or [L] of 0/1, 0 = the level is left untouched.
-    optimizer: NESTEROV (the paper's), MOMENTUM (heavy ball) or SGD.
+    optimizer: NESTEROV (the paper's), MOMENTUM (heavy ball), SGD or ADAM.
+    second_moment: float32 array like theta (ADAM only).  adam: (b1, b2, eps, weight_decay, c1, c2).
+    input_kind: COPIES, or GRADIENTS when the path buffers hold gradients instead of copies.
     """
     lib = _load()
     K = np.ascontiguousarray(modules_per_level, dtype=np.int32)
@@ -110,6 +118,13 @@ def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, 
     if level_sync is not None:
         ls = np.ascontiguousarray(level_sync, dtype=np.uint8)
         assert ls.shape == (L,)
+    ad = None
+    if adam is not None:
+        ad = np.ascontiguousarray(adam, dtype=np.float64)
+        assert ad.shape == (6,)
+    if second_moment is not None:
+        assert second_moment.dtype == np.float32 and second_moment.flags.c_contiguous
+        assert second_moment.size == total
     rc = lib.oracle_outer_sync_ex(
         L, K.ctypes.data, N.ctypes.data, P, table.ctypes.data,
         w.ctypes.data if w is not None else None,
@@ -120,6 +135,9 @@ def outer_sync(modules_per_level, level_numel, path_to_module, theta, momentum, 
         sc.ctypes.data if sc is not None else None,
         ls.ctypes.data if ls is not None else None,
         int(optimizer),
+        second_moment.ctypes.data if second_moment is not None else None,
+        ad.ctypes.data if ad is not None else None,
+        int(input_kind),
     )
     if rc != 0:
         raise ValueError("oracle_outer_sync rejected its arguments")

@@ -37,7 +37,16 @@
  *     same scheme.  Besides Nesterov (0, the paper's choice) the oracle defines heavy-ball
  *     momentum (1): m' = mu*m + Delta, theta' = theta - lr*m'; and plain SGD (2):
  *     theta' = theta - lr*Delta with the momentum buffer left as it is (lr = 1 is plain
- *     averaging of the copies).
+ *     averaging of the copies); and the Adam family (3), which covers both the adaptive
+ *     federated optimiser the paper points to in Section 2.5 and the AdamW of its fully
+ *     synchronous ablation (Section 4.3):
+ *         m' = b1*m + (1-b1)*Delta          v' = b2*v + (1-b2)*Delta^2
+ *         theta' = theta*(1 - lr*wd) - lr * (m'/c1) / (sqrt(v'/c2) + eps)
+ *     with c1 = c2 = 1 and wd = 0 for the federated form, c1 = 1-b1^t, c2 = 1-b2^t for the
+ *     bias-corrected form at step t.  m is the momentum array, v a second array.
+ *   - input_kind: 1 = the path buffers hold gradients g_i of the path's copy instead of the
+ *     copy itself (the synchronous ablation aggregates gradients module by module every step):
+ *     Delta = sum_i alpha_i * g_i; the buffers are still overwritten with cast(theta').
  *
  * Arithmetic: steps 1-3 in double, theta' and m' rounded once to float;
  * a bf16 path copy receives round-to-nearest-even of that float.
@@ -115,7 +124,10 @@ static void write_copy(void *buf, int dtype, int64_t idx, float v)
  *
  *  module_scale        [sum_l K_l] factor on each module's outer gradient, level-major, or NULL = 1
  *  level_sync          [L] 0 = leave the level untouched, or NULL = every level is synchronised
- *  optimizer           0 = Nesterov momentum, 1 = heavy-ball momentum, 2 = plain SGD
+ *  optimizer           0 = Nesterov momentum, 1 = heavy-ball momentum, 2 = plain SGD, 3 = Adam family
+ *  second_moment       float, same shape as theta; in/out (Adam family only, else NULL)
+ *  adam                {b1, b2, eps, weight decay, c1, c2} (Adam family only, else NULL)
+ *  input_kind          0 = path buffers hold copies of the modules, 1 = they hold gradients
  *
  * Returns 0, or -1 on an invalid argument.
  */
@@ -125,9 +137,12 @@ int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
                          const uint8_t *reported, double outer_lr, double outer_momentum,
                          int32_t path_dtype, float *theta, float *momentum,
                          void *const *path_ptrs, int32_t num_threads,
-                         const double *module_scale, const uint8_t *level_sync, int32_t optimizer)
+                         const double *module_scale, const uint8_t *level_sync, int32_t optimizer,
+                         float *second_moment, const double *adam, int32_t input_kind)
 {
-    if (optimizer < 0 || optimizer > 2)
+    if (optimizer < 0 || optimizer > 3 || input_kind < 0 || input_kind > 1)
+        return -1;
+    if (optimizer == 3 && (!second_moment || !adam))
         return -1;
     if (num_levels < 1 || num_paths < 1 || !modules_per_level || !level_numel ||
         !path_to_module || !theta || !momentum || !path_ptrs)
@@ -186,6 +201,7 @@ int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
 
             float *th = theta + module_base;
             float *mo = momentum + module_base;
+            float *v2 = second_moment ? second_moment + module_base : NULL;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(static) num_threads(num_threads) if (num_threads > 1)
 #endif
@@ -196,7 +212,7 @@ int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
                     double delta = 0.0;
                     for (int32_t r = 0; r < n_reporters; ++r) {
                         double x = read_copy(path_ptrs[reporters[r]], path_dtype, level_base + k);
-                        delta += alpha[r] * (t0 - x);
+                        delta += alpha[r] * (input_kind == 1 ? x : t0 - x);
                     }
                     delta *= scale;
                     double m1, t1;
@@ -206,9 +222,16 @@ int oracle_outer_sync_ex(int32_t num_levels, const int32_t *modules_per_level,
                     } else if (optimizer == 1) {   /* heavy-ball momentum */
                         m1 = outer_momentum * (double)mo[k] + delta;
                         t1 = t0 - outer_lr * m1;
-                    } else {                       /* plain SGD, momentum buffer untouched */
+                    } else if (optimizer == 2) {   /* plain SGD, momentum buffer untouched */
                         m1 = (double)mo[k];
                         t1 = t0 - outer_lr * delta;
+                    } else {                       /* Adam family */
+                        const double b1 = adam[0], b2 = adam[1], eps = adam[2], wd = adam[3];
+                        const double c1 = adam[4], c2 = adam[5];
+                        m1 = b1 * (double)mo[k] + (1.0 - b1) * delta;
+                        const double v1 = b2 * (double)v2[k] + (1.0 - b2) * delta * delta;
+                        t1 = t0 * (1.0 - outer_lr * wd) - outer_lr * (m1 / c1) / (sqrt(v1 / c2) + eps);
+                        v2[k] = (float)v1;
                     }
                     mo[k] = (float)m1;
                     new_theta = (float)t1;
@@ -234,7 +257,8 @@ int oracle_outer_sync(int32_t num_levels, const int32_t *modules_per_level,
 {
     return oracle_outer_sync_ex(num_levels, modules_per_level, level_numel, num_paths,
                                 path_to_module, path_weights, reported, outer_lr, outer_momentum,
-                                path_dtype, theta, momentum, path_ptrs, num_threads, NULL, NULL, 0);
+                                path_dtype, theta, momentum, path_ptrs, num_threads, NULL, NULL, 0, NULL, NULL,
+                                0);
 }
 
 /* number of OpenMP threads the element loop can use on this host (1 without OpenMP) */

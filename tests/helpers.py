@@ -33,7 +33,7 @@ def host_copy(problem):
 
 def run_oracle(cfg, table, theta, momentum, paths, weights=None, reported=None,
                lr=None, mu=None, num_threads=1, module_scale=None, level_sync=None,
-               optimizer=0):
+               optimizer=0, second_moment=None, adam=None, input_kind=0):
     """Oracle on copies of the given host arrays; returns (theta', m', [copies'])."""
     th = theta.copy()
     mo = momentum.copy()
@@ -43,7 +43,7 @@ def run_oracle(cfg, table, theta, momentum, paths, weights=None, reported=None,
     mu = np.float32(cfg.outer_momentum if mu is None else mu)
     oracle.outer_sync(cfg.modules_per_level, cfg.level_numel, table, th, mo, ps, dtype,
                       float(lr), float(mu), weights, reported, num_threads, module_scale, level_sync,
-                      optimizer)
+                      optimizer, second_moment, adam, input_kind)
     return th, mo, ps
 
 

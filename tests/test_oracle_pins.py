@@ -535,3 +535,76 @@ def test_heavy_ball_constant_gradient_series_and_plain_sgd():
     assert np.all(np.abs(got_th[:5] - want) <= one_ulp(want))
     with pytest.raises(ValueError):
         helpers.run_oracle(cfg, pr.table, th, mo, ps, optimizer=3)
+
+
+# ---------------------------------------------------------------------------- Adam family, gradients
+
+def test_adam_family_matches_library_adamw_on_aggregated_gradients():
+    """The synchronous variant: path buffers hold gradients, the module-wise weighted mean of them
+    drives bias-corrected AdamW.  Three steps against torch.optim.AdamW."""
+    cfg = synth.SyncConfig("dense", (1,), (97,), "f32")
+    table = np.zeros((3, 1), dtype=np.int32)
+    rng = np.random.RandomState(8)
+    theta = rng.normal(0, 0.02, 97).astype(np.float32)
+    m = np.zeros(97, dtype=np.float32)
+    v = np.zeros(97, dtype=np.float32)
+    lr, b1, b2, eps, wd = 4e-4, 0.9, 0.999, 1e-8, 0.1
+    weights = np.array([3.0, 1.0, 4.0], dtype=np.float32)
+    param = torch.nn.Parameter(torch.from_numpy(theta.copy()).double())
+    opt = torch.optim.AdamW([param], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd)
+    for t in range(1, 4):
+        grads = [rng.normal(0, 1e-2, 97).astype(np.float32) for _ in range(3)]
+        g = np.average(np.stack(grads).astype(np.float64), axis=0, weights=weights.astype(np.float64))
+        with torch.no_grad():
+            param.copy_(torch.from_numpy(theta.astype(np.float64)))
+        if t > 1:   # the oracle keeps its state in fp32: start the library step from the same state
+            opt.state[param]["exp_avg"] = torch.from_numpy(m.astype(np.float64))
+            opt.state[param]["exp_avg_sq"] = torch.from_numpy(v.astype(np.float64))
+        param.grad = torch.from_numpy(g.copy())
+        opt.step()
+        adam = (b1, b2, eps, wd, 1 - b1 ** t, 1 - b2 ** t)
+        bufs = [x.copy() for x in grads]
+        theta, m, bufs = helpers.run_oracle(cfg, table, theta, m, bufs, weights, None, lr=lr,
+                                            optimizer=oracle.ADAM, second_moment=v, adam=adam,
+                                            input_kind=oracle.GRADIENTS)
+        want = param.detach().numpy()
+        assert np.all(np.abs(theta - want) <= one_ulp(want))
+        np.testing.assert_allclose(m, opt.state[param]["exp_avg"].numpy(), rtol=2e-7, atol=1e-45)
+        np.testing.assert_allclose(v, opt.state[param]["exp_avg_sq"].numpy(), rtol=2e-7, atol=1e-45)
+        for b in bufs:      # the buffers now hold the new parameters
+            np.testing.assert_array_equal(b, theta)
+
+
+def test_federated_adam_closed_forms_on_outer_gradients():
+    """No bias correction, no decay: from m = v = 0 the first step is
+    lr*(1-b1)*Delta / (sqrt(1-b2)*|Delta| + tau); with b1 = b2 = 0 it is lr*Delta/(|Delta| + tau);
+    a constant outer gradient drives the step towards lr*g/(|g| + tau)."""
+    cfg = tiny_cfg((1,), (6,))
+    table = synth.path_table(cfg.modules_per_level)
+    theta = np.array([1.0, -2.0, 0.5, 3.0, -0.25, 8.0], dtype=np.float32)
+    delta = np.array([0.5, -0.25, 0.125, 1.0, -2.0, 0.0], dtype=np.float32)
+    zeros = np.zeros(6, dtype=np.float32)
+    lr, tau = 0.1, 1e-3
+    for b1, b2 in ((0.9, 0.99), (0.0, 0.0)):
+        v = zeros.copy()
+        th, m, _ = helpers.run_oracle(cfg, table, theta, zeros, [theta - delta], lr=lr,
+                                      optimizer=oracle.ADAM, second_moment=v, adam=(b1, b2, tau, 0, 1, 1))
+        d = delta.astype(np.float64)
+        want = theta - lr * (1 - b1) * d / (np.sqrt(1 - b2) * np.abs(d) + tau)
+        assert np.all(np.abs(th - want) <= one_ulp(want))
+        np.testing.assert_allclose(m, (1 - b1) * d, rtol=2e-7)
+        np.testing.assert_allclose(v, (1 - b2) * d * d, rtol=2e-7)
+    th, m, v = theta.copy(), zeros.copy(), zeros.copy()
+    for _ in range(400):
+        prev = th
+        th, m, _ = helpers.run_oracle(cfg, table, th, m, [th - delta], lr=lr, optimizer=oracle.ADAM,
+                                      second_moment=v, adam=(0.9, 0.9, tau, 0, 1, 1))
+    d = delta.astype(np.float64)
+    np.testing.assert_allclose(prev - th, lr * d / (np.abs(d) + tau), rtol=1e-4, atol=1e-6)
+    # gradients as inputs with plain SGD: theta' = theta - lr * weighted mean of the gradients
+    g = [np.full(6, 2.0, np.float32), np.full(6, 4.0, np.float32)]
+    th, _, _ = helpers.run_oracle(cfg, np.zeros((2, 1), np.int32), theta, zeros, g, lr=0.5,
+                                  optimizer=oracle.SGD, input_kind=oracle.GRADIENTS)
+    np.testing.assert_array_equal(th, theta - np.float32(1.5))
+    with pytest.raises(ValueError):
+        helpers.run_oracle(cfg, table, theta, zeros, [theta.copy()], optimizer=oracle.ADAM)
