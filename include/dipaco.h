@@ -153,7 +153,7 @@ int dipaco_set_weights(dipaco_ctx *ctx, const float *path_weights);
 int dipaco_set_module_scale(dipaco_ctx *ctx, const float *module_scale);
 
 /*
- * Levels that take no part in the exchange (Section 4.1: in the models with path-specific
+ * Levels that take no part in the exchange (Section 4.2: in the models with path-specific
  * modules some blocks stay local to their path): host [L], 0 = theta, momentum and every copy
  * of the level's modules are left untouched; NULL = every level is synchronised.
  */

@@ -24,12 +24,12 @@
  *   4. every path of S(l,e), reporting or not, receives cast(theta')
  *      (Section 2.5: the new global vector is re-dispatched to all workers).
  *
- * Two options of Section 2.7 / Section 4.1, off by default:
+ * Options of Sections 2.5, 2.7, 4.2 and 4.5, off by default:
  *   - module_scale: the outer gradient of module (l,e) is multiplied by s(l,e) before the
  *     optimiser step, Delta <- s * Delta ("Outer Gradient Norm Rescaling": the paper rescales
  *     by the square root of the number of paths through the module; the caller supplies s, so
  *     whether that means sqrt(P) or 1/sqrt(P) is the caller's reading).
- *   - level_sync: a level flagged 0 takes no part in the exchange (Section 4.1 keeps some
+ *   - level_sync: a level flagged 0 takes no part in the exchange (Section 4.2 keeps some
  *     blocks of the path-specific models local to their path): theta, momentum and every copy
  *     of its modules are left untouched.
  *
@@ -39,7 +39,7 @@
  *     theta' = theta - lr*Delta with the momentum buffer left as it is (lr = 1 is plain
  *     averaging of the copies); and the Adam family (3), which covers both the adaptive
  *     federated optimiser the paper points to in Section 2.5 and the AdamW of its fully
- *     synchronous ablation (Section 4.3):
+ *     synchronous ablation (Section 4.5):
  *         m' = b1*m + (1-b1)*Delta          v' = b2*v + (1-b2)*Delta^2
  *         theta' = theta*(1 - lr*wd) - lr * (m'/c1) / (sqrt(v'/c2) + eps)
  *     with c1 = c2 = 1 and wd = 0 for the federated form, c1 = 1-b1^t, c2 = 1-b2^t for the
