@@ -66,6 +66,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-chunked", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true")
     return ap.parse_args()
 
 
@@ -389,6 +390,10 @@ def run_ours(args):
                      "frac_of_nominal_8tbs": achieved / 8000.0},
     }
 
+    # ---- the same launch with the optional features switched on (resident mode, rank 0)
+    if not args.no_variants and rank == 0:
+        result["variants"] = run_variants(args, cfg, problem, make_ctx, ptrs, alg_bytes)
+
     # ---- the same workload walked in chunks of paths (device resident)
     if not args.no_chunked and cfg.chunk_paths > 0 and rank == 0:
         ctx = make_ctx(cfg.chunk_paths)
@@ -423,6 +428,51 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def run_variants(args, cfg, problem, make_ctx, ptrs, alg_bytes):
+    """ms per synchronisation with the optional features on: gradient rescaling by sqrt(paths per
+    module), heavy-ball and SGD outer optimisers, and the Adam family (one more fp32 state array:
+    8 more bytes per module parameter)."""
+    import torch
+    from paper_2403_10616_b200 import binding as B
+    steps = max(3, min(args.steps, 8))
+    out = {}
+
+    def timed(ctx):
+        fn = lambda: B.dipaco_outer_sync(ctx, problem.theta.data_ptr(), problem.momentum.data_ptr(),
+                                         ptrs, problem.reported)
+        for _ in range(2):
+            fn()
+        ms, _ = time_steps(fn, steps, 1)
+        ok = B.dipaco_device_status(ctx) == B.DIPACO_OK
+        B.dipaco_destroy(ctx)
+        return ms if ok else None
+
+    ctx = make_ctx(0)
+    scale = np.concatenate([np.full(k, np.sqrt(cfg.num_paths / k), dtype=np.float32)
+                            for k in cfg.modules_per_level])
+    B.dipaco_set_module_scale(ctx, scale)
+    out["rescaled_sqrt_paths_ms"] = timed(ctx)
+    for name, opt in (("heavy_ball_ms", B.DIPACO_OPT_MOMENTUM), ("sgd_ms", B.DIPACO_OPT_SGD)):
+        ctx = make_ctx(0)
+        B.dipaco_set_optimizer(ctx, opt)
+        out[name] = timed(ctx)
+    try:
+        second = torch.zeros_like(problem.theta)
+    except RuntimeError:
+        second = None
+    if second is not None:
+        ctx = make_ctx(0)
+        B.dipaco_set_adam(ctx, second.data_ptr(), 0.9, 0.99, 1e-3, 0.0, 0)
+        ms = timed(ctx)
+        out["adam_ms"] = ms
+        if ms:
+            out["adam_gbs"] = (alg_bytes + 8 * cfg.module_params) / (ms * 1e-3) / 1e9
+        del second
+        torch.cuda.empty_cache()
+    out["steps"] = steps
+    return out
 
 
 def host_memory_available():

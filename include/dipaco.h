@@ -59,7 +59,14 @@ enum {
 enum {
     DIPACO_OPT_NESTEROV = 0, /* m' = mu*m + Delta; theta' = theta - lr*(Delta + mu*m')   (the paper's) */
     DIPACO_OPT_MOMENTUM = 1, /* m' = mu*m + Delta; theta' = theta - lr*m'                (heavy ball)  */
-    DIPACO_OPT_SGD = 2       /* theta' = theta - lr*Delta; momentum left as it is (lr = 1: averaging)   */
+    DIPACO_OPT_SGD = 2,      /* theta' = theta - lr*Delta; momentum left as it is (lr = 1: averaging)   */
+    DIPACO_OPT_ADAM = 3      /* Adam family, configured by dipaco_set_adam                              */
+};
+
+/* what the path buffers hold on entry, for dipaco_set_input_kind */
+enum {
+    DIPACO_INPUT_COPIES = 0,   /* each path's copy x_i of its modules: Delta = sum c_i (theta - x_i)  */
+    DIPACO_INPUT_GRADIENTS = 1 /* each path's gradient g_i of its modules: Delta = sum c_i g_i         */
 };
 
 /* kernel selection for dipaco_set_kernel */
@@ -166,6 +173,29 @@ int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync);
 int dipaco_set_optimizer(dipaco_ctx *ctx, int32_t optimizer);
 
 /*
+ * Adam-family optimiser.  It covers the adaptive federated optimisers that Section 2.5 names as
+ * alternatives (step = 0: no bias correction, eps plays the role of their adaptivity constant)
+ * and the AdamW of the fully synchronous ablation of Section 4.5 (step = t >= 1: bias-corrected,
+ * decoupled weight decay).  With Delta the module's outer gradient, the `momentum` argument of
+ * the sync calls as first moment m and second_moment as v:
+ *     m' = b1*m + (1-b1)*Delta        v' = b2*v + (1-b2)*Delta^2
+ *     theta' = theta*(1 - lr*weight_decay) - lr * (m'/c1) / (sqrt(v'/c2) + eps)
+ *     c1 = 1 - b1^step, c2 = 1 - b2^step   (both 1 when step = 0)
+ * second_moment: device, fp32, same layout as theta, caller-owned, in/out.  0 <= b1, b2 < 1,
+ * eps >= 0.  Selects DIPACO_OPT_ADAM; call again to advance `step`.  The outer_momentum given at
+ * create is not used.  Not available through dipaco_outer_sync_host (DIPACO_ESTATE).
+ */
+int dipaco_set_adam(dipaco_ctx *ctx, float *second_moment, float beta1, float beta2, float eps,
+                    float weight_decay, int32_t step);
+
+/*
+ * What the path buffers hold on entry (DIPACO_INPUT_*).  With gradients the reduction is the
+ * module-by-module gradient aggregation of Section 4.5; the buffers are still overwritten with
+ * cast(theta') on exit, so after the call every path holds the new parameters of its modules.
+ */
+int dipaco_set_input_kind(dipaco_ctx *ctx, int32_t input_kind);
+
+/*
  * Sharded executor (Section 3.3, "Sharded Outer Optimization Executor": modules, and the
  * parameters inside a module, are independent, so the update can be split over executors with no
  * exchange between them).  This context then owns slab shard_index of shard_count of EVERY
@@ -186,7 +216,9 @@ int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
  * 256 threads * units * 16 bytes) and the number of theta/momentum/result tile buffers (2..4;
  * more of them help modules with few contributors).  0 keeps a value.  A depth that does not fit
  * the shared memory of the chosen layout is rejected with DIPACO_EINVAL and nothing changes;
- * result buffers beyond two are dropped at launch if they would leave fewer than 6 stages.
+ * result buffers beyond two are dropped at launch while they would leave the ring shallower than a
+ * launch of that mix of modules needs (10 stages when most elements have 8 or more contributors,
+ * 6 otherwise).
  */
 int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
                       int32_t units_per_thread, int32_t io_slots);

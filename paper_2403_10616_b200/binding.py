@@ -32,6 +32,10 @@ DIPACO_STATIC_MAX_NUMEL = 4 * 1024 * 1024
 DIPACO_OPT_NESTEROV = 0
 DIPACO_OPT_MOMENTUM = 1
 DIPACO_OPT_SGD = 2
+DIPACO_OPT_ADAM = 3
+
+DIPACO_INPUT_COPIES = 0
+DIPACO_INPUT_GRADIENTS = 1
 
 DIPACO_KERNEL_AUTO = 0
 DIPACO_KERNEL_VECTOR = 1
@@ -44,7 +48,8 @@ EXPORTS = [
     "dipaco_device_status", "dipaco_launch_count", "dipaco_plan_module", "dipaco_plan_offsets",
     "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
     "dipaco_set_host_unit_bytes", "dipaco_plan_traffic", "dipaco_set_module_scale",
-    "dipaco_set_level_sync", "dipaco_set_shard", "dipaco_set_optimizer",
+    "dipaco_set_level_sync", "dipaco_set_shard", "dipaco_set_optimizer", "dipaco_set_adam",
+    "dipaco_set_input_kind",
 ]
 
 _lib = None
@@ -82,6 +87,8 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_level_sync.argtypes = [vp, vp]
     lib.dipaco_set_shard.argtypes = [vp, i32, i32]
     lib.dipaco_set_optimizer.argtypes = [vp, i32]
+    lib.dipaco_set_adam.argtypes = [vp, vp, f32, f32, f32, f32, i32]
+    lib.dipaco_set_input_kind.argtypes = [vp, i32]
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32, i32]
     lib.dipaco_device_status.argtypes = [vp]
@@ -211,6 +218,16 @@ def dipaco_set_level_sync(ctx, level_sync) -> None:
 
 def dipaco_set_optimizer(ctx, optimizer: int) -> None:
     _check(load().dipaco_set_optimizer(ctx, int(optimizer)), "dipaco_set_optimizer")
+
+
+def dipaco_set_adam(ctx, second_moment_ptr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0,
+                    step=0) -> None:
+    _check(load().dipaco_set_adam(ctx, second_moment_ptr, float(beta1), float(beta2), float(eps),
+                                  float(weight_decay), int(step)), "dipaco_set_adam")
+
+
+def dipaco_set_input_kind(ctx, input_kind: int) -> None:
+    _check(load().dipaco_set_input_kind(ctx, int(input_kind)), "dipaco_set_input_kind")
 
 
 def dipaco_set_shard(ctx, shard_index: int, shard_count: int) -> None:

@@ -38,6 +38,7 @@ struct PackedLaunch {
     int io_arrays = 2;
     bool aligned_kernel_is_vector = false;
     int num_passes = 0, total_items = 0;  // dynamic scheduling of the bulk-copy kernel
+    double mean_contributors = 0.0;       // per element of the bulk range
 };
 
 struct HostMode;  // state of dipaco_outer_sync_host (host_mode.inl)
@@ -48,6 +49,11 @@ struct dipaco_ctx {
     Grid grid;
     float lr = 0.f, mu = 0.f;
     int optimizer = DIPACO_OPT_NESTEROV;
+    int input_kind = DIPACO_INPUT_COPIES;
+    // Adam family
+    float *second_moment = nullptr;
+    double adam_b1 = 0.9, adam_b2 = 0.999, adam_eps = 1e-8, adam_wd = 0.0;
+    int adam_step = 0;  // 0 = no bias correction
     int dtype = DIPACO_F32;
     int elem_size = 4;
     int device = -1;
@@ -181,6 +187,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
         bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
                        ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
+        if (ctx->optimizer == DIPACO_OPT_ADAM)
+            aligned = aligned && ((uintptr_t)(ctx->second_moment + m.theta_off) % 16 == 0);
         pd.contrib_begin = (int)contribs.size();
         for (size_t j = 0; j < sp.contributors.size(); ++j) {
             char *base = static_cast<char *>(lookup.get(sp.contributors[j]));
@@ -228,8 +236,10 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     const bool vector_kernel = ctx->kernel == DIPACO_KERNEL_VECTOR;
     int bulk_ctas = ctx->sm_count * (vector_kernel ? 8 : ctx->ctas_per_sm);
     int64_t bulk_tiles = 0, rag_tiles = 0;
-    double bulk_bytes = 0.0;
+    double bulk_bytes = 0.0, contrib_elems = 0.0, bulk_elems = 0.0;
     for (size_t i = 0; i < specs.size(); ++i) {
+        contrib_elems += (double)specs[i].contributors.size() * (double)(bulk_end[i] - bulk_begin[i]);
+        bulk_elems += (double)(bulk_end[i] - bulk_begin[i]);
         bulk_tiles += (bulk_end[i] - bulk_begin[i] + tile - 1) / tile;
         bulk_bytes += pass_cost_per_elem(specs[i], es) * (double)(bulk_end[i] - bulk_begin[i]);
         rag_tiles += (rag_end[i] - rag_begin[i] + RAGGED_TILE - 1) / RAGGED_TILE;
@@ -277,10 +287,11 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     out.rag_first_off = append(rag_first.data(), rag_first.size() * sizeof(int32_t));
     out.bulk_ctas = bulk_ctas;
     out.rag_ctas = rag_ctas;
-    out.io_arrays = any_partial ? 3 : 2;
+    out.io_arrays = (any_partial ? 3 : 2) + (ctx->optimizer == DIPACO_OPT_ADAM ? 1 : 0);
     out.aligned_kernel_is_vector = vector_kernel;
     out.num_passes = (int)passes.size();
     out.total_items = (int)total_items;
+    out.mean_contributors = bulk_elems > 0.0 ? contrib_elems / bulk_elems : 0.0;
     return DIPACO_OK;
 }
 
@@ -347,11 +358,16 @@ int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages,
     return cudaGetLastError() == cudaSuccess ? DIPACO_OK : DIPACO_ECUDA;
 }
 
-int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays, cudaStream_t stream)
+int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays,
+                double mean_contributors, cudaStream_t stream)
 {
-    // more result buffers only while the copy ring keeps a useful depth
+    // Shared memory is split between the ring of path tiles and the theta/momentum/result
+    // buffers.  Launches dominated by many-contributor modules need the ring depth (10 stages
+    // measured best), launches with few contributors per module need the extra buffers.
+    const int wanted = ctx->stages > 0 ? std::min(ctx->stages, 10) : 10;
+    const int min_stages = mean_contributors >= 8.0 ? wanted : std::min(wanted, 6);
     int io_slots = ctx->io_slots;
-    while (io_slots > 2 && pick_stages(ctx, io_arrays, io_slots) < 6) --io_slots;
+    while (io_slots > 2 && pick_stages(ctx, io_arrays, io_slots) < min_stages) --io_slots;
     const int stages = pick_stages(ctx, io_arrays, io_slots);
     if (stages < 2) return DIPACO_EINVAL;
     const size_t smem = bulk_smem_bytes(ctx, stages, io_arrays, io_slots);
@@ -378,9 +394,21 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
     lp.passes = reinterpret_cast<const PassDev *>(base + pl.passes_off);
     lp.contribs = reinterpret_cast<const ContribDev *>(base + pl.contribs_off);
     lp.members = reinterpret_cast<void *const *>(base + pl.members_off);
-    lp.lr = ctx->lr;
-    lp.mu = ctx->mu;
-    lp.optimizer = ctx->optimizer;
+    const bool adam = ctx->optimizer == DIPACO_OPT_ADAM;
+    lp.rule.lr = ctx->lr;
+    lp.rule.mu = ctx->mu;
+    lp.rule.optimizer = ctx->optimizer;
+    lp.rule.b1 = (float)ctx->adam_b1;
+    lp.rule.one_minus_b1 = (float)(1.0 - ctx->adam_b1);
+    lp.rule.b2 = (float)ctx->adam_b2;
+    lp.rule.one_minus_b2 = (float)(1.0 - ctx->adam_b2);
+    lp.rule.eps = (float)ctx->adam_eps;
+    lp.rule.decay = (float)(1.0 - (double)ctx->lr * ctx->adam_wd);
+    lp.rule.inv_c1 = ctx->adam_step > 0 ? (float)(1.0 / (1.0 - std::pow(ctx->adam_b1, ctx->adam_step))) : 1.0f;
+    lp.rule.inv_c2 = ctx->adam_step > 0 ? (float)(1.0 / (1.0 - std::pow(ctx->adam_b2, ctx->adam_step))) : 1.0f;
+    lp.second_moment = adam ? ctx->second_moment : nullptr;
+    lp.input_kind = ctx->input_kind;
+    lp.v_index = pl.io_arrays - 1;
     lp.error_word = ctx->error_word;
     lp.num_passes = pl.num_passes;
     lp.total_items = pl.total_items;
@@ -396,7 +424,7 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
                 sync_direct_kernel<float, 8><<<pl.bulk_ctas, 256, 0, stream>>>(lp);
             if (cudaGetLastError() != cudaSuccess) rc = DIPACO_ECUDA;
         } else {
-            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, stream);
+            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, pl.mean_contributors, stream);
         }
         if (rc != DIPACO_OK) return rc;
         ++ctx->launches;
@@ -585,9 +613,38 @@ int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync)
 
 int dipaco_set_optimizer(dipaco_ctx *ctx, int32_t optimizer)
 {
-    if (!ctx || optimizer < DIPACO_OPT_NESTEROV || optimizer > DIPACO_OPT_SGD) return DIPACO_EINVAL;
+    if (!ctx || optimizer < DIPACO_OPT_NESTEROV || optimizer > DIPACO_OPT_ADAM) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    if (optimizer == DIPACO_OPT_ADAM && !ctx->second_moment) return DIPACO_ESTATE;  // dipaco_set_adam first
     ctx->optimizer = optimizer;
+    ctx->grid.second_moment = optimizer == DIPACO_OPT_ADAM;
+    return DIPACO_OK;
+}
+
+int dipaco_set_adam(dipaco_ctx *ctx, float *second_moment, float beta1, float beta2, float eps,
+                    float weight_decay, int32_t step)
+{
+    if (!ctx || !second_moment || step < 0) return DIPACO_EINVAL;
+    if (!(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f)) return DIPACO_EINVAL;
+    if (!(eps >= 0.0f) || !std::isfinite(eps) || !std::isfinite(weight_decay)) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ctx->second_moment = second_moment;
+    ctx->adam_b1 = beta1;
+    ctx->adam_b2 = beta2;
+    ctx->adam_eps = eps;
+    ctx->adam_wd = weight_decay;
+    ctx->adam_step = step;
+    ctx->optimizer = DIPACO_OPT_ADAM;
+    ctx->grid.second_moment = true;
+    return DIPACO_OK;
+}
+
+int dipaco_set_input_kind(dipaco_ctx *ctx, int32_t input_kind)
+{
+    if (!ctx || (input_kind != DIPACO_INPUT_COPIES && input_kind != DIPACO_INPUT_GRADIENTS))
+        return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ctx->input_kind = input_kind;
     return DIPACO_OK;
 }
 
@@ -623,7 +680,7 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
     if (units_per_thread) ctx->units = units_per_thread;
     ctx->stages = 0;
     // chunked contexts stage a third fp32 tile (the partial sum) per buffer
-    const int io_arrays = ctx->grid.num_chunks > 1 ? 3 : 2;
+    const int io_arrays = (ctx->grid.num_chunks > 1 ? 3 : 2) + (ctx->optimizer == DIPACO_OPT_ADAM ? 1 : 0);
     const bool fits = pick_stages(ctx, io_arrays, 2) >= 2 && (!stages || stages <= pick_stages(ctx, io_arrays, 2));
     if (!fits) {
         ctx->ctas_per_sm = old_ctas;
@@ -772,6 +829,7 @@ int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_h
     if (ctx->device < 0) return DIPACO_ENODEV;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
     if (ctx->grid.chunk_paths <= 0) return DIPACO_ESTATE;
+    if (ctx->optimizer == DIPACO_OPT_ADAM) return DIPACO_ESTATE;  // v lives on the device only
     if (!valid_ptr_array(path_ptrs_host, ctx->grid.P)) return DIPACO_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DIPACO_ECUDA;

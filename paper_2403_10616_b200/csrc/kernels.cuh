@@ -46,6 +46,18 @@ struct SegmentDev {
     long long begin, end;  // element range inside the module
 };
 
+enum : int { KOPT_NESTEROV = 0, KOPT_MOMENTUM = 1, KOPT_SGD = 2, KOPT_ADAM = 3 };
+
+struct UpdateRule {
+    float lr, mu;
+    int optimizer;  // KOPT_*
+    // Adam family (constants rounded once from double on the host)
+    float b1, one_minus_b1, b2, one_minus_b2;
+    float eps;
+    float decay;    // 1 - lr * weight_decay
+    float inv_c1, inv_c2;  // reciprocals of the bias corrections 1 - b^t, or 1
+};
+
 struct LaunchParams {
     float *theta;
     float *momentum;
@@ -55,8 +67,10 @@ struct LaunchParams {
     void *const *members;  // start of the module's slot inside each member path copy
     const SegmentDev *segs;
     const int *cta_first;  // [gridDim.x + 1]
-    float lr, mu;
-    int optimizer;  // KOPT_*
+    UpdateRule rule;       // outer optimiser and its constants
+    float *second_moment;  // Adam family only: v, same layout as theta
+    int input_kind;        // 0: path buffers hold copies of the modules, 1: they hold gradients
+    int v_index;           // bulk-copy kernel: which fp32 tile of a buffer carries v
     int *error_word;
     // bulk-copy kernel only
     int num_passes;
@@ -69,30 +83,40 @@ struct LaunchParams {
 // The arithmetic, written once (sync_accumulate, sync_update).  Explicit intrinsics: no contraction or reassociation choices
 // are left to the compiler, so every kernel family rounds identically.
 
-__device__ __forceinline__ float sync_accumulate(float acc, float c, float theta, float x)
+__device__ __forceinline__ float sync_accumulate(float acc, float c, float theta, float x, int input_kind)
 {
-    // acc + c * (theta - x): one term of the outer gradient (Algorithm 1, outer-gradient line)
-    return __fmaf_rn(c, __fsub_rn(theta, x), acc);
+    // acc + c * (theta - x): one term of the outer gradient (Algorithm 1, outer-gradient line);
+    // acc + c * x when the buffers hold gradients (Section 4.5, module-wise gradient aggregation)
+    const float d = input_kind ? x : __fsub_rn(theta, x);
+    return __fmaf_rn(c, d, acc);
 }
 
-enum : int { KOPT_NESTEROV = 0, KOPT_MOMENTUM = 1, KOPT_SGD = 2 };
-
-__device__ __forceinline__ void sync_update(float theta, float m, float sum, float scale, float lr,
-                                            float mu, int optimizer, float &theta_new, float &m_new)
+__device__ __forceinline__ void sync_update(float theta, float m, float &v, float sum, float scale,
+                                            const UpdateRule &r, float &theta_new, float &m_new)
 {
     // Delta = scale * sum, then the outer optimiser step:
     //   Nesterov   m' = mu*m + Delta ; theta' = theta - lr*(Delta + mu*m')
     //   heavy ball m' = mu*m + Delta ; theta' = theta - lr*m'
     //   SGD        m' = m            ; theta' = theta - lr*Delta
+    //   Adam       m' = b1*m + (1-b1)*Delta ; v' = b2*v + (1-b2)*Delta^2
+    //              theta' = theta*decay - lr * (m'*inv_c1) / (sqrt(v'*inv_c2) + eps)
     const float delta = __fmul_rn(scale, sum);  // exact when scale == 1
-    if (optimizer == KOPT_SGD) {
-        m_new = m;
-        theta_new = __fmaf_rn(-lr, delta, theta);
+    if (r.optimizer == KOPT_ADAM) {
+        m_new = __fmaf_rn(r.b1, m, __fmul_rn(r.one_minus_b1, delta));
+        v = __fmaf_rn(r.b2, v, __fmul_rn(r.one_minus_b2, __fmul_rn(delta, delta)));
+        const float denom = __fadd_rn(__fsqrt_rn(__fmul_rn(v, r.inv_c2)), r.eps);
+        const float step = __fdiv_rn(__fmul_rn(m_new, r.inv_c1), denom);
+        theta_new = __fmaf_rn(-r.lr, step, __fmul_rn(theta, r.decay));
         return;
     }
-    m_new = __fmaf_rn(mu, m, delta);
-    const float g = optimizer == KOPT_NESTEROV ? __fmaf_rn(mu, m_new, delta) : m_new;
-    theta_new = __fmaf_rn(-lr, g, theta);
+    if (r.optimizer == KOPT_SGD) {
+        m_new = m;
+        theta_new = __fmaf_rn(-r.lr, delta, theta);
+        return;
+    }
+    m_new = __fmaf_rn(r.mu, m, delta);
+    const float g = r.optimizer == KOPT_NESTEROV ? __fmaf_rn(r.mu, m_new, delta) : m_new;
+    theta_new = __fmaf_rn(-r.lr, g, theta);
 }
 
 template <typename T> struct PathIO;
@@ -186,12 +210,12 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
                         x[u] = PathIO<PathT>::load(static_cast<const PathT *>(c.src) + k);
                     }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) acc[0] = sync_accumulate(acc[0], cf[u], th[0], x[u]);
+                    for (int u = 0; u < 4; ++u) acc[0] = sync_accumulate(acc[0], cf[u], th[0], x[u], p.input_kind);
                 }
                 for (; j < pass.contrib_count; ++j) {
                     const ContribDev c = contribs[j];
                     const float x = PathIO<PathT>::load(static_cast<const PathT *>(c.src) + k);
-                    acc[0] = sync_accumulate(acc[0], c.coeff, th[0], x);
+                    acc[0] = sync_accumulate(acc[0], c.coeff, th[0], x, p.input_kind);
                 }
             } else {
                 constexpr int UE = Unit<PathT>::UE;
@@ -236,7 +260,7 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
 #pragma unroll
                                 for (int i = 0; i < UE; ++i)
                                     acc[u * UE + i] =
-                                        sync_accumulate(acc[u * UE + i], coeff[b], th[u * UE + i], x[i]);
+                                        sync_accumulate(acc[u * UE + i], coeff[b], th[u * UE + i], x[i], p.input_kind);
                             }
                         }
                     }
@@ -264,12 +288,21 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
                         mo[v] = t.x; mo[v + 1] = t.y; mo[v + 2] = t.z; mo[v + 3] = t.w;
                     }
                 }
+                const bool adam = p.rule.optimizer == KOPT_ADAM;
+                float *second = p.second_moment + pass.theta_off;
+                float sm[VEC];
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) sm[v] = adam ? second[k + v] : 0.0f;
 #pragma unroll
                 for (int v = 0; v < VEC; ++v) {
                     float t1, m1;
-                    sync_update(th[v], mo[v], acc[v], pass.scale, p.lr, p.mu, p.optimizer, t1, m1);
+                    sync_update(th[v], mo[v], sm[v], acc[v], pass.scale, p.rule, t1, m1);
                     th[v] = t1;
                     mo[v] = m1;
+                }
+                if (adam) {
+#pragma unroll
+                    for (int v = 0; v < VEC; ++v) second[k + v] = sm[v];
                 }
                 if constexpr (VEC == 1) {
                     theta[k] = th[0];
@@ -520,7 +553,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
     auto io_tile = [&](int b, int which) -> float * {
         return reinterpret_cast<float *>(io + ((size_t)b * io_arrays + which) * F32_TILE_BYTES);
     };
-    // io tile roles: 0 = theta (becomes theta'), 1 = momentum (becomes m'), 2 = partial sum
+    // io tile roles: 0 = theta (becomes theta'), 1 = momentum (becomes m'), 2 = partial sum (chunked
+    // contexts), v_index = second moment (Adam family)
     auto cast_tile = [&](int b) -> unsigned char * {
         return NEED_CAST_TILE ? cast_tiles + (size_t)b * STAGE_BYTES
                               : reinterpret_cast<unsigned char *>(io_tile(b, 0));
@@ -583,7 +617,9 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                 if (ok) {
                     const unsigned f32_bytes = n * 4u;
                     unsigned bytes = f32_bytes;
+                    const bool adam = (pass.flags & KPASS_UPDATE) && p.rule.optimizer == KOPT_ADAM;
                     if (pass.flags & KPASS_UPDATE) bytes += f32_bytes;
+                    if (adam) bytes += f32_bytes;
                     if (pass.flags & KPASS_PARTIAL_IN) bytes += f32_bytes;
                     ptx::mbar_arrive_expect_tx(&sh->io_full[b], bytes);
                     ptx::bulk_load(io_tile(b, 0), p.theta + pass.theta_off + k0, f32_bytes,
@@ -594,6 +630,9 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                     if (pass.flags & KPASS_PARTIAL_IN)
                         ptx::bulk_load(io_tile(b, 2), p.partial + pass.partial_off + k0, f32_bytes,
                                        &sh->io_full[b]);
+                    if (adam)
+                        ptx::bulk_load(io_tile(b, p.v_index), p.second_moment + pass.theta_off + k0,
+                                       f32_bytes, &sh->io_full[b]);
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -648,6 +687,9 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                 if (pass.flags & KPASS_UPDATE) {
                     ptx::bulk_store(p.theta + pass.theta_off + k0, io_tile(b, 0), n * 4u);
                     ptx::bulk_store(p.momentum + pass.theta_off + k0, io_tile(b, 1), n * 4u);
+                    if (p.rule.optimizer == KOPT_ADAM)
+                        ptx::bulk_store(p.second_moment + pass.theta_off + k0, io_tile(b, p.v_index),
+                                        n * 4u);
                 }
                 if (pass.flags & KPASS_PARTIAL_OUT)
                     ptx::bulk_store(p.partial + pass.partial_off + k0, io_tile(b, 2), n * 4u);
@@ -717,7 +759,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                     Unit<PathT>::widen(raw[u], x);
 #pragma unroll
                     for (int i = 0; i < UE; ++i)
-                        acc[u * UE + i] = sync_accumulate(acc[u * UE + i], c, th[u * UE + i], x[i]);
+                        acc[u * UE + i] = sync_accumulate(acc[u * UE + i], c, th[u * UE + i], x[i], p.input_kind);
                 }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&sh->empty[s]);
@@ -739,6 +781,8 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
             }
             if (pass.flags & KPASS_UPDATE) {
                 float *mo_tile = io_tile(b, 1);
+                const bool adam = p.rule.optimizer == KOPT_ADAM;
+                float *v_tile = io_tile(b, adam ? p.v_index : 1);
 #pragma unroll
                 for (int u = 0; u < NU; ++u) {
                     const int e0 = (u * BULK_COMPUTE_THREADS + ct) * UE;
@@ -746,11 +790,19 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                     for (int v = 0; v < UE; v += 4) {
                         const float4 m4 = *reinterpret_cast<const float4 *>(mo_tile + e0 + v);
                         const float mo[4] = {m4.x, m4.y, m4.z, m4.w};
+                        float sm[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                        if (adam) {
+                            const float4 v4 = *reinterpret_cast<const float4 *>(v_tile + e0 + v);
+                            sm[0] = v4.x; sm[1] = v4.y; sm[2] = v4.z; sm[3] = v4.w;
+                        }
                         float m1[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            sync_update(th[u * UE + v + i], mo[i], acc[u * UE + v + i], pass.scale, p.lr,
-                                        p.mu, p.optimizer, th[u * UE + v + i], m1[i]);
+                            sync_update(th[u * UE + v + i], mo[i], sm[i], acc[u * UE + v + i], pass.scale,
+                                        p.rule, th[u * UE + v + i], m1[i]);
+                        if (adam)
+                            *reinterpret_cast<float4 *>(v_tile + e0 + v) =
+                                make_float4(sm[0], sm[1], sm[2], sm[3]);
                         *reinterpret_cast<float4 *>(mo_tile + e0 + v) =
                             make_float4(m1[0], m1[1], m1[2], m1[3]);
                         *reinterpret_cast<float4 *>(th_tile + e0 + v) =

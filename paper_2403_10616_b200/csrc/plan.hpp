@@ -40,6 +40,7 @@ struct Grid {
     int chunk_paths = 0, num_chunks = 1;
     int64_t scratch_elems = 0;
     int shard_index = 0, shard_count = 1;  // this context owns one slab of every module
+    bool second_moment = false;            // the optimiser keeps a second state array (Adam family)
 
     int module_id(int l, int e) const { return level_first[l] + e; }
     bool synced(const ModuleGeom &m) const { return level_sync.empty() || level_sync[(size_t)m.level]; }
@@ -158,6 +159,7 @@ struct PassSpec {
     std::vector<int> members;      // path ids written in this launch
     int64_t begin = 0, end = -1;   // element range of the module ([0, numel) when end < 0)
     float scale = 1.0f;            // factor on the finished outer gradient (used with PASS_UPDATE)
+    bool second_moment = false;    // the update also reads and writes v (Adam family)
 };
 
 // Resident mode: one launch covers every module completely.
@@ -174,6 +176,7 @@ inline void plan_resident(const Grid &g, const std::vector<ModuleCoeffs> &mc,
         if (p.begin >= p.end) continue;
         p.scale = g.scale_of(id);
         p.flags = mc[id].update ? PASS_UPDATE : 0;
+        p.second_moment = g.second_moment;
         p.contributors = mc[id].contributors;
         p.coeff = mc[id].coeff;
         p.members = m.members;
@@ -206,6 +209,7 @@ inline void plan_accumulate(const Grid &g, const std::vector<ModuleCoeffs> &mc, 
         if (c > first) p.flags |= PASS_PARTIAL_IN;
         if (c == last) {
             p.flags |= PASS_UPDATE;
+            p.second_moment = g.second_moment;
             for (int i : m.members)
                 if (g.chunk_of(i) == c) p.members.push_back(i);
         } else {
@@ -251,6 +255,7 @@ inline double pass_cost_per_elem(const PassSpec &p, int elem_size)
     double c = 4.0; // theta read
     c += (double)elem_size * (double)(p.contributors.size() + p.members.size());
     if (p.flags & PASS_UPDATE) c += 12.0;      // momentum read, theta' and m' written
+    if ((p.flags & PASS_UPDATE) && p.second_moment) c += 8.0;  // v read and written
     if (p.flags & PASS_PARTIAL_IN) c += 4.0;
     if (p.flags & PASS_PARTIAL_OUT) c += 4.0;
     return c;

@@ -48,11 +48,15 @@ __global__ void __launch_bounds__(256) static_accumulate_kernel(StaticAccumulate
         float acc = (a.flags & KPASS_PARTIAL_IN) ? a.partial[k] : 0.0f;
         for (int j = 0; j < a.count; ++j)
             acc = sync_accumulate(acc, a.coeff[j], th,
-                                  PathIO<PathT>::load(static_cast<const PathT *>(a.src[j]) + k));
+                                  PathIO<PathT>::load(static_cast<const PathT *>(a.src[j]) + k), 0);
         if (a.flags & KPASS_PARTIAL_OUT) a.partial[k] = acc;
         if (a.flags & KPASS_UPDATE) {
-            float t1, m1;
-            sync_update(th, a.momentum[k], acc, 1.0f, a.lr, a.mu, KOPT_NESTEROV, t1, m1);
+            float t1, m1, unused = 0.0f;
+            UpdateRule rule = {};
+            rule.lr = a.lr;
+            rule.mu = a.mu;
+            rule.optimizer = KOPT_NESTEROV;
+            sync_update(th, a.momentum[k], unused, acc, 1.0f, rule, t1, m1);
             a.theta[k] = t1;
             a.momentum[k] = m1;
         }

@@ -530,3 +530,70 @@ def test_calls_run_on_the_callers_stream():
     assert abs(total - want) <= 1e-4 * (1 + abs(want))
     err = (theta.double() - ref[0].double()).abs()
     assert bool((err <= 1e-6 * (1 + ref[0].double().abs())).all())
+
+
+@pytest.mark.parametrize("variant", ["federated", "adamw_gradients"])
+@pytest.mark.parametrize("chunk,kernel", [(0, B.DIPACO_KERNEL_AUTO), (32, B.DIPACO_KERNEL_AUTO),
+                                          (0, B.DIPACO_KERNEL_VECTOR), (5, B.DIPACO_KERNEL_SCALAR)])
+def test_adam_family_and_gradient_inputs_match_the_oracle(variant, chunk, kernel):
+    base = synth.CONFIGS["grid16x16-masked"]
+    cfg = dataclass_replace(base.scaled((4096 + 72, 2 * 4096 + 8, 4096 + 1003)), momentum_std=1e-4)
+    pr = synth.make_problem(cfg, DEV)
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(3)
+    second = torch.empty_like(pr.theta).normal_(0, 1e-4, generator=gen).abs_()
+    if variant == "adamw_gradients":
+        # the buffers hold gradients, not copies; two consecutive steps of bias-corrected AdamW
+        for p in pr.paths:
+            p.copy_(torch.empty(p.numel(), device=DEV).normal_(0, 1e-2, generator=gen))
+        lr, adam_args, steps, kind = 4e-4, (0.9, 0.999, 1e-8, 0.1), (1, 2), B.DIPACO_INPUT_GRADIENTS
+    else:
+        lr, adam_args, steps, kind = 0.1, (0.9, 0.99, 1e-3, 0.0), (0,), B.DIPACO_INPUT_COPIES
+    theta, momentum, paths = clone_problem(pr)
+    v = second.clone()
+    th, mo, ps = host_state((theta, momentum, paths))
+    v_host = helpers.tensor_to_numpy(v)
+    code = B.DIPACO_BF16
+    ctx = B.dipaco_create(cfg.modules_per_level, cfg.level_numel, pr.table, pr.weights, np.float32(lr),
+                          np.float32(0.9), code, chunk, 0)
+    B.dipaco_set_kernel(ctx, kernel)
+    B.dipaco_set_input_kind(ctx, kind)
+    for step in steps:
+        B.dipaco_set_adam(ctx, v.data_ptr(), *adam_args, step)
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths],
+                            pr.reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        b1, b2, eps, wd = [float(np.float32(x)) for x in adam_args]
+        c1 = 1 - b1 ** step if step else 1.0
+        c2 = 1 - b2 ** step if step else 1.0
+        th, mo, ps = helpers.run_oracle(cfg, pr.table, th, mo, ps, pr.weights, pr.reported, lr=lr,
+                                        num_threads=8, optimizer=3, second_moment=v_host,
+                                        adam=(b1, b2, eps, wd, c1, c2), input_kind=int(kind))
+        for got, want in ((theta, th), (momentum, mo), (v, v_host)):
+            g = helpers.tensor_to_numpy(got).astype(np.float64)
+            assert np.all(np.abs(g - want) <= 1e-6 * (1.0 + np.abs(want.astype(np.float64))))
+        for i in range(0, cfg.num_paths, 9):
+            assert_bf16_close(helpers.tensor_to_numpy(paths[i]), ps[i])
+        if len(steps) > 1:
+            # next step: fresh gradients in the buffers, oracle continues from the device state
+            th, mo = helpers.tensor_to_numpy(theta), helpers.tensor_to_numpy(momentum)
+            v_host = helpers.tensor_to_numpy(v)
+            for i, p in enumerate(paths):
+                p.copy_(torch.empty(p.numel(), device=DEV).normal_(0, 1e-2, generator=gen))
+                ps[i] = helpers.tensor_to_numpy(p)
+    # the host-buffer entry point has no second-moment argument
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_outer_sync_host(ctx, 16, 16, [16] * cfg.num_paths)
+    assert e.value.status == B.DIPACO_ESTATE
+    B.dipaco_destroy(ctx)
+
+
+def test_adam_needs_its_second_moment_first():
+    pr = synth.make_problem(synth.CONFIGS["grid2x2"], DEV)
+    ctx = make_ctx(pr)
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_set_optimizer(ctx, B.DIPACO_OPT_ADAM)
+    assert e.value.status == B.DIPACO_ESTATE
+    with pytest.raises(B.DipacoError):
+        B.dipaco_set_adam(ctx, pr.theta.data_ptr(), 1.0, 0.9, 1e-8, 0.0, 0)
+    B.dipaco_destroy(ctx)
