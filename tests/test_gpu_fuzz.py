@@ -50,13 +50,16 @@ def random_case(seed):
             int(rng.randint(0, 6))],
         "scale": rng.choice([0.5, 1.0, 2.0, 3.0], size=sum(K)).astype(np.float32) if rng.rand() < 0.4 else None,
         "level_sync": (rng.rand(L) > 0.3).astype(np.uint8) if rng.rand() < 0.3 else None,
-        "optimizer": int(rng.choice([0, 0, 1, 2])),
+        "optimizer": int(rng.choice([0, 0, 1, 2, 3])),
+        "adam": (float(rng.choice([0.0, 0.5, 0.9])), float(rng.choice([0.0, 0.9, 0.999])), 1e-3,
+                 float(rng.choice([0.0, 0.1])), int(rng.choice([0, 1, 7]))),
+        "input_kind": int(rng.rand() < 0.25),
         "misalign": bool(rng.rand() < 0.2),
     }
     return K, numel, table, dtype, weights, reported, opts
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(64))
 def test_random_structure_matches_the_oracle(seed):
     K, numel, table, dtype, weights, reported, opts = random_case(seed)
     cfg = synth.SyncConfig("fuzz%d" % seed, tuple(K), tuple(numel), dtype, momentum_std=1e-4, seed=seed)
@@ -92,7 +95,18 @@ def test_random_structure_matches_the_oracle(seed):
         assert exc.status == B.DIPACO_EINVAL
     B.dipaco_set_module_scale(ctx, opts["scale"])
     B.dipaco_set_level_sync(ctx, opts["level_sync"])
-    B.dipaco_set_optimizer(ctx, opts["optimizer"])
+    second = torch.empty_like(theta).normal_(0, 1e-4, generator=gen).abs_()
+    v_host = helpers.tensor_to_numpy(second)
+    adam = None
+    if opts["optimizer"] == 3:
+        b1, b2, eps, wd, step = opts["adam"]
+        B.dipaco_set_adam(ctx, second.data_ptr(), b1, b2, eps, wd, step)
+        f = lambda x: float(np.float32(x))
+        adam = (f(b1), f(b2), f(eps), f(wd), 1 - f(b1) ** step if step else 1.0,
+                1 - f(b2) ** step if step else 1.0)
+    else:
+        B.dipaco_set_optimizer(ctx, opts["optimizer"])
+    B.dipaco_set_input_kind(ctx, opts["input_kind"])
     B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths], reported)
     assert B.dipaco_device_status(ctx) == B.DIPACO_OK
     B.dipaco_destroy(ctx)
@@ -101,8 +115,11 @@ def test_random_structure_matches_the_oracle(seed):
     want_th, want_mo, want_ps = helpers.run_oracle(cfg, pr.table, *before, weights, reported,
                                                    num_threads=4, module_scale=scale64,
                                                    level_sync=opts["level_sync"],
-                                                   optimizer=opts["optimizer"])
-    for got, want in ((helpers.tensor_to_numpy(theta), want_th), (helpers.tensor_to_numpy(momentum), want_mo)):
+                                                   optimizer=opts["optimizer"],
+                                                   second_moment=v_host if adam else None, adam=adam,
+                                                   input_kind=opts["input_kind"])
+    for got, want in ((helpers.tensor_to_numpy(theta), want_th), (helpers.tensor_to_numpy(momentum), want_mo),
+                      (helpers.tensor_to_numpy(second), v_host)):
         err = np.abs(got.astype(np.float64) - want.astype(np.float64))
         assert np.all(err <= 1e-6 * (1.0 + np.abs(want.astype(np.float64))))
     for p, want in zip(paths, want_ps):
