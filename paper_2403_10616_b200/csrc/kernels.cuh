@@ -1,13 +1,14 @@
 // Device code of the outer synchronisation (DiPaCo, Algorithm 1, outer loop + re-dispatch).
 //
-// Three kernel families share one arithmetic definition (sync_math below), so they give
-// bitwise identical results:
+// Three kernel families share one arithmetic definition (sync_accumulate, sync_update), so they
+// give bitwise identical results:
 //   sync_direct_kernel<PathT,1>   one element per thread, any alignment (ragged tails, odd offsets)
 //   sync_direct_kernel<PathT,8>   128-bit register loads/stores on 16-byte aligned full tiles
-//   sync_bulk_kernel<PathT,NU>    persistent, warp-specialised: one warp streams tiles into a
-//                                 shared-memory ring with bulk async copies (TMA, 1-D), eight
-//                                 warps reduce + apply Nesterov, one warp scatters the result
-//                                 tile to every path with bulk stores from shared memory.
+//   sync_bulk_kernel<PathT,NU>    persistent, warp-specialised: a scheduler warp draws work items
+//                                 from a counter, one warp streams tiles into a shared-memory
+//                                 ring with bulk async copies (TMA, 1-D), eight warps reduce and
+//                                 apply the optimiser step, one warp scatters the result tile to
+//                                 every path with bulk stores from shared memory.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -80,8 +81,8 @@ struct LaunchParams {
 };
 
 // ------------------------------------------------------------------------------------------
-// The arithmetic, written once (sync_accumulate, sync_update).  Explicit intrinsics: no contraction or reassociation choices
-// are left to the compiler, so every kernel family rounds identically.
+// The arithmetic, written once (sync_accumulate, sync_update).  Explicit intrinsics: no contraction
+// or reassociation choices are left to the compiler, so every kernel family rounds identically.
 
 __device__ __forceinline__ float sync_accumulate(float acc, float c, float theta, float x, int input_kind)
 {
