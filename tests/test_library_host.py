@@ -246,3 +246,15 @@ def test_shards_partition_the_planned_traffic():
         with pytest.raises(B.DipacoError):
             B.dipaco_set_shard(ctx, *bad)
     B.dipaco_destroy(ctx)
+
+
+def test_a_c99_program_can_use_the_library(tmp_path):
+    """The header compiles as C and a plain C caller links against the shared library."""
+    import subprocess
+    exe = str(tmp_path / "plan_from_c")
+    src = os.path.join(ROOT, "tests", "c", "plan_from_c.c")
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), src,
+                           "-o", exe, "-L", libdir, "-ldipaco", "-Wl,-rpath," + libdir])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.strip() == "ok", out.stdout + out.stderr
