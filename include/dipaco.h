@@ -183,7 +183,8 @@ int dipaco_set_optimizer(dipaco_ctx *ctx, int32_t optimizer);
  *     c1 = 1 - b1^step, c2 = 1 - b2^step   (both 1 when step = 0)
  * second_moment: device, fp32, same layout as theta, caller-owned, in/out.  0 <= b1, b2 < 1,
  * eps >= 0.  Selects DIPACO_OPT_ADAM; call again to advance `step`.  The outer_momentum given at
- * create is not used.  Not available through dipaco_outer_sync_host (DIPACO_ESTATE).
+ * create is not used.  second_moment lives where theta lives: a device array for
+ * dipaco_outer_sync and the chunk API, a host array for dipaco_outer_sync_host.
  */
 int dipaco_set_adam(dipaco_ctx *ctx, float *second_moment, float beta1, float beta2, float eps,
                     float weight_decay, int32_t step);

@@ -52,6 +52,7 @@ struct dipaco_ctx {
     int input_kind = DIPACO_INPUT_COPIES;
     // Adam family
     float *second_moment = nullptr;
+    float *second_moment_staged = nullptr;  // host mode: device copy that the kernels use instead
     double adam_b1 = 0.9, adam_b2 = 0.999, adam_eps = 1e-8, adam_wd = 0.0;
     int adam_step = 0;  // 0 = no bias correction
     int dtype = DIPACO_F32;
@@ -187,8 +188,10 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
         bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
                        ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
-        if (ctx->optimizer == DIPACO_OPT_ADAM)
-            aligned = aligned && ((uintptr_t)(ctx->second_moment + m.theta_off) % 16 == 0);
+        if (ctx->optimizer == DIPACO_OPT_ADAM) {
+            const float *v = ctx->second_moment_staged ? ctx->second_moment_staged : ctx->second_moment;
+            aligned = aligned && ((uintptr_t)(v + m.theta_off) % 16 == 0);
+        }
         pd.contrib_begin = (int)contribs.size();
         for (size_t j = 0; j < sp.contributors.size(); ++j) {
             char *base = static_cast<char *>(lookup.get(sp.contributors[j]));
@@ -406,7 +409,8 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
     lp.rule.decay = (float)(1.0 - (double)ctx->lr * ctx->adam_wd);
     lp.rule.inv_c1 = ctx->adam_step > 0 ? (float)(1.0 / (1.0 - std::pow(ctx->adam_b1, ctx->adam_step))) : 1.0f;
     lp.rule.inv_c2 = ctx->adam_step > 0 ? (float)(1.0 / (1.0 - std::pow(ctx->adam_b2, ctx->adam_step))) : 1.0f;
-    lp.second_moment = adam ? ctx->second_moment : nullptr;
+    lp.second_moment = !adam ? nullptr
+                             : (ctx->second_moment_staged ? ctx->second_moment_staged : ctx->second_moment);
     lp.input_kind = ctx->input_kind;
     lp.v_index = pl.io_arrays - 1;
     lp.error_word = ctx->error_word;
@@ -829,7 +833,6 @@ int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_h
     if (ctx->device < 0) return DIPACO_ENODEV;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
     if (ctx->grid.chunk_paths <= 0) return DIPACO_ESTATE;
-    if (ctx->optimizer == DIPACO_OPT_ADAM) return DIPACO_ESTATE;  // v lives on the device only
     if (!valid_ptr_array(path_ptrs_host, ctx->grid.P)) return DIPACO_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DIPACO_ECUDA;

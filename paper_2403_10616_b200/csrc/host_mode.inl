@@ -18,6 +18,7 @@ namespace {
 
 struct HostMode {
     float *theta_d = nullptr, *momentum_d = nullptr;  // full module state on the device
+    float *second_d = nullptr;                        // second moment (Adam family), on demand
     char *stage_in[2] = {nullptr, nullptr};           // staged pieces of path copies
     char *stage_out[2] = {nullptr, nullptr};          // cast(theta') of the unit (bf16 paths)
     size_t stage_in_bytes = 0, stage_out_bytes = 0;
@@ -36,6 +37,7 @@ void host_mode_release(dipaco_ctx *ctx)
     if (h->out_stream) cudaStreamSynchronize(h->out_stream);
     if (h->theta_d) cudaFree(h->theta_d);
     if (h->momentum_d) cudaFree(h->momentum_d);
+    if (h->second_d) cudaFree(h->second_d);
     for (int b = 0; b < 2; ++b) {
         if (h->stage_in[b]) cudaFree(h->stage_in[b]);
         if (h->stage_out[b]) cudaFree(h->stage_out[b]);
@@ -108,6 +110,19 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
     const int es = ctx->elem_size;
     const int64_t tile = tile_elems(ctx);
     compute_all_coeffs(ctx, reported);
+    // Adam family: the caller's second moment is a host array here; the kernels get a device copy
+    const bool adam = ctx->optimizer == DIPACO_OPT_ADAM;
+    float *second_host = ctx->second_moment;
+    if (adam && !h->second_d &&
+        cudaMalloc(&h->second_d, std::max<size_t>((size_t)g.module_params * sizeof(float), 16)) != cudaSuccess) {
+        cudaGetLastError();
+        return DIPACO_ENOMEM;
+    }
+    struct StagedSecondMoment {  // the kernels see the device copy for the duration of this call
+        dipaco_ctx *c;
+        StagedSecondMoment(dipaco_ctx *ctx_, float *p) : c(ctx_) { c->second_moment_staged = p; }
+        ~StagedSecondMoment() { c->second_moment_staged = nullptr; }
+    } staged(ctx, adam ? h->second_d : nullptr);
 
     // the side streams must not run ahead of work queued earlier on the caller's stream
     if (cudaEventRecord(h->main_ready, stream) != cudaSuccess ||
@@ -151,6 +166,10 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
                 return DIPACO_ECUDA;
             if (mc.update &&
                 cudaMemcpyAsync(h->momentum_d + m.theta_off + a, momentum_host + m.theta_off + a, fbytes,
+                                cudaMemcpyHostToDevice, h->in_stream) != cudaSuccess)
+                return DIPACO_ECUDA;
+            if (mc.update && adam &&
+                cudaMemcpyAsync(h->second_d + m.theta_off + a, second_host + m.theta_off + a, fbytes,
                                 cudaMemcpyHostToDevice, h->in_stream) != cudaSuccess)
                 return DIPACO_ECUDA;
             for (size_t j = 0; j < ncon; ++j) {
@@ -200,6 +219,10 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
                                     cudaMemcpyDeviceToHost, h->out_stream) != cudaSuccess ||
                     cudaMemcpyAsync(momentum_host + m.theta_off + a, h->momentum_d + m.theta_off + a,
                                     fbytes, cudaMemcpyDeviceToHost, h->out_stream) != cudaSuccess)
+                    return DIPACO_ECUDA;
+                if (adam &&
+                    cudaMemcpyAsync(second_host + m.theta_off + a, h->second_d + m.theta_off + a, fbytes,
+                                    cudaMemcpyDeviceToHost, h->out_stream) != cudaSuccess)
                     return DIPACO_ECUDA;
             }
             const char *out_src = es != 4 ? h->stage_out[buf]

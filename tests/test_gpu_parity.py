@@ -581,10 +581,6 @@ def test_adam_family_and_gradient_inputs_match_the_oracle(variant, chunk, kernel
             for i, p in enumerate(paths):
                 p.copy_(torch.empty(p.numel(), device=DEV).normal_(0, 1e-2, generator=gen))
                 ps[i] = helpers.tensor_to_numpy(p)
-    # the host-buffer entry point has no second-moment argument
-    with pytest.raises(B.DipacoError) as e:
-        B.dipaco_outer_sync_host(ctx, 16, 16, [16] * cfg.num_paths)
-    assert e.value.status == B.DIPACO_ESTATE
     B.dipaco_destroy(ctx)
 
 
@@ -597,3 +593,28 @@ def test_adam_needs_its_second_moment_first():
     with pytest.raises(B.DipacoError):
         B.dipaco_set_adam(ctx, pr.theta.data_ptr(), 1.0, 0.9, 1e-8, 0.0, 0)
     B.dipaco_destroy(ctx)
+
+
+def test_adam_family_through_the_host_buffer_entry_point():
+    """theta, momentum, the second moment and the path copies all live in host memory; the result
+    is bitwise the device-resident one."""
+    base = synth.CONFIGS["grid16x16-masked"]
+    cfg = dataclass_replace(base.scaled((4096 + 72, 2 * 4096 + 8, 4096 + 1003)), momentum_std=1e-4)
+    pr = synth.make_problem(cfg, "cpu")
+    second = torch.empty_like(pr.theta).normal_(0, 1e-4).abs_()
+    host = [t.clone().pin_memory() for t in (pr.theta, pr.momentum, second)]
+    host_paths = [p.clone().pin_memory() for p in pr.paths]
+    dev = [t.to(DEV) for t in (pr.theta, pr.momentum, second)]
+    dev_paths = [p.to(DEV) for p in pr.paths]
+    for where, (theta, momentum, v), paths in (("host", host, host_paths), ("device", dev, dev_paths)):
+        ctx = make_ctx(pr, chunk_paths=32 if where == "host" else 0)
+        B.dipaco_set_adam(ctx, v.data_ptr(), 0.9, 0.99, 1e-3, 0.01, 3)
+        fn = B.dipaco_outer_sync_host if where == "host" else B.dipaco_outer_sync
+        fn(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths], pr.reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        B.dipaco_destroy(ctx)
+    for a, b in zip(host, dev):
+        assert torch.equal(a.view(torch.int32), b.cpu().view(torch.int32))
+    for a, b in zip(host_paths, dev_paths):
+        assert torch.equal(a.view(torch.int16), b.cpu().view(torch.int16))
+    assert not torch.equal(host[2], second)
