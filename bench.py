@@ -34,17 +34,23 @@ REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the referen
 # DRAM traffic of the bulk-copy kernel from the ncu capture summarised under profiles/ (small case of
 # the same workload, 2e6 parameters per level): dram__bytes_read.sum + dram__bytes_write.sum divided
 # by the algorithmic bytes of that launch.  Traffic grows with the number of tiles, so the full-size
-# figure is this ratio times the algorithmic bytes.  Only valid for the kernel source it was taken
-# from: the digest below is checked and "traffic" is null after any change to the kernels.
+# figure is this ratio times the algorithmic bytes.  Only valid for the sources it was taken from
+# (the kernels, the launch code that picks tiles, stages and work items, and the planner): their
+# digest is checked and "traffic" is null after any change to them.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9917
-NCU_CAPTURE_KERNELS_SHA256 = "228ef41efc8b5bc82345ec9971ad706a0974b353e6be729c039a5ac81c0f441d"
+NCU_CAPTURE_SOURCES = ("kernels.cuh", "dipaco.cu", "plan.hpp")
+NCU_CAPTURE_SOURCES_SHA256 = "unset"
+NCU_CAPTURE_COMMAND = ("ncu --set full --clock-control none -k regex:sync_bulk_kernel -s 3 -c 3 "
+                       "python bench.py --level-numel 2000000 --steps 3 --warmup 3 --no-e2e "
+                       "--no-chunked --no-cpu-baseline --no-variants --no-other-workloads")
 
 
-def kernels_digest():
+def sources_digest():
     import hashlib
     h = hashlib.sha256()
-    with open(os.path.join(ROOT, "paper_2403_10616_b200", "csrc", "kernels.cuh"), "rb") as f:
-        h.update(f.read())
+    for name in NCU_CAPTURE_SOURCES:
+        with open(os.path.join(ROOT, "paper_2403_10616_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
     return h.hexdigest()
 
 
@@ -57,15 +63,22 @@ def parse_args():
     ap.add_argument("--workload", default="grid16x16")
     ap.add_argument("--level-numel", type=int, default=0,
                     help="override the parameters per level (smaller runs for profiling)")
-    ap.add_argument("--mode", default="resident", choices=["resident", "chunked", "adam"],
-                    help="what the main timed leg runs (the metric is quoted on 'resident'; the "
-                         "others exist to profile the chunk walk and the Adam-family step)")
+    ap.add_argument("--mode", default="resident", choices=["resident", "chunked", "adam", "sharded"],
+                    help="what the main timed leg runs (the metric is quoted on 'resident'; 'chunked' "
+                         "and 'adam' exist to profile the chunk walk and the Adam-family step; "
+                         "'sharded' splits the ONE workload over the ranks, rank r updating slab r "
+                         "of every module with no exchange: strong scaling)")
     ap.add_argument("--kernel", default="auto", choices=["auto", "vector", "scalar"])
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--units", type=int, default=0)
     ap.add_argument("--io-slots", type=int, default=0)
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--host-unit-mb", type=int, default=0,
+                    help="cap on the upload of one streamed unit of the host-buffer leg (0 = default)")
+    ap.add_argument("--items-per-cta", type=int, default=0)
+    ap.add_argument("--item-kb", type=int, default=0)
+    ap.add_argument("--no-other-workloads", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-chunked", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -317,6 +330,23 @@ def run_ours(args):
     B.load()
 
     cfg = workload_config(args)
+    whole_cfg, whole_plan = cfg, None
+    if args.mode == "sharded":
+        # Section 3.3, sharded executor: rank r owns slab r of every module of the ONE workload and
+        # holds only that slab of theta, momentum and of every path copy (compact layout).  The
+        # slab is itself a grid with smaller modules; its synthetic values are drawn per rank.
+        import dataclasses
+        code_w = B.DIPACO_BF16 if cfg.path_dtype == "bf16" else B.DIPACO_F32
+        whole_plan = B.dipaco_create(cfg.modules_per_level, cfg.level_numel,
+                                     synth.path_table(cfg.modules_per_level), synth.path_weights(cfg),
+                                     np.float32(cfg.outer_lr), np.float32(cfg.outer_momentum), code_w,
+                                     0, device=-1)
+        slabs = []
+        for l in range(cfg.num_levels):
+            a, b = B.dipaco_plan_shard(whole_plan, rank, world, l)
+            slabs.append(b - a)
+        cfg = dataclasses.replace(cfg.scaled(slabs, name="%s-shard%dof%d" % (cfg.name, rank, world)),
+                                  seed=cfg.seed + rank)
     need = cfg.path_params * (2 if cfg.path_dtype == "bf16" else 4) + 8 * cfg.module_params
     free, _total = torch.cuda.mem_get_info(device)
     if need * 1.02 > free:
@@ -329,24 +359,34 @@ def run_ours(args):
               "scalar": B.DIPACO_KERNEL_SCALAR}[args.kernel]
     code = B.DIPACO_BF16 if cfg.path_dtype == "bf16" else B.DIPACO_F32
 
-    def make_ctx(chunk_paths):
-        ctx = B.dipaco_create(cfg.modules_per_level, cfg.level_numel, problem.table, problem.weights,
-                              np.float32(cfg.outer_lr), np.float32(cfg.outer_momentum), code,
-                              chunk_paths, local)
+    def tune(ctx):
         B.dipaco_set_kernel(ctx, kernel)
         B.dipaco_set_tuning(ctx, args.ctas_per_sm, args.stages, args.units, args.io_slots)
+        B.dipaco_set_work_items(ctx, args.item_kb * 1024, args.items_per_cta)
         return ctx
 
+    def make_ctx(chunk_paths):
+        return tune(B.dipaco_create(cfg.modules_per_level, cfg.level_numel, problem.table,
+                                    problem.weights, np.float32(cfg.outer_lr),
+                                    np.float32(cfg.outer_momentum), code, chunk_paths, local))
+
     # ---- resident one-pass mode: the headline value (--mode selects another leg for profiling)
-    ctx = make_ctx(cfg.chunk_paths if args.mode == "chunked" else 0)
+    if args.mode == "sharded":
+        ctx = tune(B.dipaco_create_shard(whole_plan, rank, world, local))
+        B.dipaco_destroy(whole_plan)
+    else:
+        ctx = make_ctx(cfg.chunk_paths if args.mode == "chunked" else 0)
     second = None
     if args.mode == "adam":
         second = torch.zeros_like(problem.theta)
         B.dipaco_set_adam(ctx, second.data_ptr(), 0.9, 0.99, 1e-3, 0.0, 0)
 
+    ptr_arr = B.ptr_array(ptrs)
+    theta_ptr, momentum_ptr = problem.theta.data_ptr(), problem.momentum.data_ptr()
+    stream_handle = int(torch.cuda.current_stream().cuda_stream)
+
     def step():
-        B.dipaco_outer_sync(ctx, problem.theta.data_ptr(), problem.momentum.data_ptr(), ptrs,
-                            problem.reported)
+        B.dipaco_outer_sync(ctx, theta_ptr, momentum_ptr, ptr_arr, problem.reported, stream_handle)
 
     for _ in range(max(args.warmup, 0)):
         step()
@@ -376,17 +416,22 @@ def run_ours(args):
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True,
+        "scaling": "strong" if args.mode == "sharded" else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": cfg.name, "levels": list(cfg.modules_per_level),
-            "level_numel": list(cfg.level_numel), "paths": cfg.num_paths,
-            "path_dtype": cfg.path_dtype,
+            "workload": whole_cfg.name, "levels": list(whole_cfg.modules_per_level),
+            "level_numel": list(whole_cfg.level_numel), "paths": whole_cfg.num_paths,
+            "path_dtype": whole_cfg.path_dtype,
             "mode": {"resident": "resident one-pass (all path copies in HBM)",
                      "chunked": "chunks of %d paths, partial sums carried (all chunks in HBM)" % cfg.chunk_paths,
-                     "adam": "resident one-pass, Adam-family outer optimiser"}[args.mode],
-            "l2": "inputs (%.1f GB) exceed L2, no flush between steps" % (need / 1e9),
-            "parallelism": "replicas only" if world > 1 else "1 GPU",
+                     "adam": "resident one-pass, Adam-family outer optimiser",
+                     "sharded": "resident one-pass on this rank's slab of every module (compact "
+                                "layout, no exchange between ranks)"}[args.mode],
+            "l2": "inputs (%.1f GB per GPU) exceed L2, no flush between steps" % (need / 1e9),
+            "parallelism": ("1 GPU" if world == 1 else
+                            "one problem split over %d ranks by parameter slab, no collective" % world
+                            if args.mode == "sharded" else "replicas only"),
             "kernel": args.kernel,
         },
         "clocks": clocks,
@@ -396,7 +441,8 @@ def run_ours(args):
                      "frac": achieved / peak,
                      "traffic": (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes
                                  if args.kernel == "auto" and cfg.name == "grid16x16" and args.mode == "resident"
-                                 and kernels_digest() == NCU_CAPTURE_KERNELS_SHA256 else None),
+                                 and sources_digest() == NCU_CAPTURE_SOURCES_SHA256 else None),
+                     "traffic_from": NCU_CAPTURE_COMMAND,
                      "peak_kind": "of " + peak_kind,
                      "kernel": "sync_bulk_kernel" if args.kernel == "auto" else "sync_direct_kernel",
                      "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": ms_call,
@@ -404,20 +450,18 @@ def run_ours(args):
     }
 
     # ---- the same launch with the optional features switched on (resident mode, rank 0)
-    if not args.no_variants and rank == 0:
+    if not args.no_variants and rank == 0 and args.mode != "sharded":
         result["variants"] = run_variants(args, cfg, problem, make_ctx, ptrs, alg_bytes)
 
     # ---- the same workload walked in chunks of paths (device resident)
-    if not args.no_chunked and cfg.chunk_paths > 0 and rank == 0:
+    if not args.no_chunked and cfg.chunk_paths > 0 and rank == 0 and args.mode != "sharded":
         ctx = make_ctx(cfg.chunk_paths)
+        chunk_step = lambda: B.dipaco_outer_sync(ctx, theta_ptr, momentum_ptr, ptr_arr, problem.reported,
+                                                 stream_handle)
         for _ in range(max(args.warmup, 1)):
-            step_ctx = ctx
-            B.dipaco_outer_sync(step_ctx, problem.theta.data_ptr(), problem.momentum.data_ptr(), ptrs,
-                                problem.reported)
+            chunk_step()
         before = B.dipaco_launch_count(ctx)
-        ms_c, _ = time_steps(lambda: B.dipaco_outer_sync(ctx, problem.theta.data_ptr(),
-                                                         problem.momentum.data_ptr(), ptrs,
-                                                         problem.reported), args.steps, 1)
+        ms_c, _ = time_steps(chunk_step, args.steps, 1)
         moved, n_launch = B.dipaco_plan_traffic(ctx, problem.reported)
         result["chunked"] = {"chunk_paths": cfg.chunk_paths, "ms_per_step": ms_c,
                              "bytes_moved_by_construction": moved,
@@ -435,6 +479,15 @@ def run_ours(args):
     # ---- end to end through the host-buffer entry point
     if not args.no_e2e:
         result["e2e"] = run_e2e(args, cfg, problem, make_ctx, world, device)
+
+    # ---- the other workloads of the method's evaluation, same kernel and defaults (N = 1 only:
+    # with more ranks the other GPUs would idle meanwhile)
+    if not args.no_other_workloads and world == 1 and args.mode == "resident" and not args.level_numel:
+        problem.paths.clear()
+        problem.storage = None
+        problem.theta = problem.momentum = None
+        torch.cuda.empty_cache()
+        result["other_workloads"] = run_other_workloads(args, cfg.name, tune, local, peak)
 
     if rank == 0:
         print(json.dumps(result))
@@ -485,6 +538,77 @@ def run_variants(args, cfg, problem, make_ctx, ptrs, alg_bytes):
         del second
         torch.cuda.empty_cache()
     out["steps"] = steps
+    return out
+
+
+def run_other_workloads(args, skip_name, tune, local, peak):
+    """ms per synchronisation of the remaining workloads (resident one-pass, default kernel).  Each
+    timed region lasts at least 0.6 s so that the clock sampler sees it; the 2x2 grid (9 MB, L2
+    resident) is a latency figure, reported in microseconds per call."""
+    import math
+    import torch
+    from paper_2403_10616_b200 import binding as B
+    from paper_2403_10616_b200 import synth
+    out = []
+    for name in ("grid2x2", "grid4x4", "grid16x16-masked", "grid4x4x4x4"):
+        if name == skip_name:
+            continue
+        cfg = synth.CONFIGS[name]
+        es = 2 if cfg.path_dtype == "bf16" else 4
+        need = cfg.path_params * es + 8 * cfg.module_params
+        torch.cuda.empty_cache()
+        free, _ = torch.cuda.mem_get_info()
+        if need * 1.02 > free:
+            out.append({"workload": name, "skipped": "needs %.1f GB, %.1f GB free" % (need / 1e9, free / 1e9)})
+            continue
+        problem = synth.make_problem(cfg, "cuda:%d" % local)
+        code = B.DIPACO_BF16 if cfg.path_dtype == "bf16" else B.DIPACO_F32
+        ctx = tune(B.dipaco_create(cfg.modules_per_level, cfg.level_numel, problem.table, problem.weights,
+                                   np.float32(cfg.outer_lr), np.float32(cfg.outer_momentum), code, 0, local))
+        arr = B.ptr_array([p.data_ptr() for p in problem.paths])
+        th, mo = problem.theta.data_ptr(), problem.momentum.data_ptr()
+        handle = int(torch.cuda.current_stream().cuda_stream)
+        fn = lambda: B.dipaco_outer_sync(ctx, th, mo, arr, problem.reported, handle)
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(10):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        probe_ms = max(a.elapsed_time(b) / 10, 1e-3)
+        steps = int(min(max(math.ceil(600.0 / probe_ms), 20), 200000))
+        sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                               else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+        sampler.wait_first_sample()
+        torch.cuda.synchronize()
+        sampler.mark_start()
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        sampler.mark_end()
+        clocks = sampler.stop()
+        ms = a.elapsed_time(b) / steps
+        ok = B.dipaco_device_status(ctx) == B.DIPACO_OK
+        B.dipaco_destroy(ctx)
+        alg = synth.algorithmic_bytes(cfg, problem.reported)
+        entry = {"workload": name, "steps": steps, "ms_per_step": ms, "status_ok": ok,
+                 "value": cfg.path_params / (ms * 1e-3), "unit": UNIT,
+                 "algorithmic_bytes": alg, "clocks": clocks}
+        if need < 126e6:
+            entry["us_per_call"] = ms * 1e3
+            entry["note"] = "fits in L2: launch latency, not a roofline point"
+        else:
+            gbs = alg / (ms * 1e-3) / 1e9
+            entry.update({"algorithmic_gbs": gbs, "frac_of_peak": gbs / peak,
+                          "frac_of_nominal_8tbs": gbs / 8000.0})
+        out.append(entry)
+        del problem, arr
+        torch.cuda.empty_cache()
     return out
 
 
@@ -555,13 +679,18 @@ def run_e2e(args, cfg, problem, make_ctx, world, device):
     def step():
         B.dipaco_outer_sync_host(ctx, theta_h.data_ptr(), mom_h.data_ptr(), hptrs, problem.reported)
 
+    if args.host_unit_mb:
+        B.dipaco_set_host_unit_bytes(ctx, args.host_unit_mb << 20)
     step()   # warm-up: allocates the staging buffers
     steps = max(1, args.e2e_steps)
     barrier(world)
     torch.cuda.synchronize()
+    per_step = []
     t0 = time.perf_counter()
     for _ in range(steps):
-        step()
+        t1 = time.perf_counter()
+        step()          # synchronous: returns when the host buffers hold the result
+        per_step.append((time.perf_counter() - t1) * 1e3)
     torch.cuda.synchronize()
     dt_ms = (time.perf_counter() - t0) * 1e3 / steps
     barrier(world)
@@ -569,6 +698,7 @@ def run_e2e(args, cfg, problem, make_ctx, world, device):
     n_rep = small.num_paths if problem.reported is None else int(problem.reported.sum())
     B.dipaco_destroy(ctx)
     out = {"value": units / (ms_max * 1e-3), "unit": UNIT, "ms_per_step": ms_max, "steps": steps,
+           "ms_per_step_min": min(per_step), "ms_per_step_mean": sum(per_step) / len(per_step),
            "h2d_bytes_per_step": 8 * small.module_params + n_rep * small.params_per_path * es,
            "d2h_bytes_per_step": 8 * small.module_params + small.num_paths * small.params_per_path * es,
            "api": "dipaco_outer_sync_host, pinned host buffers, slab-ordered streaming, staging "

@@ -104,8 +104,11 @@ int dipaco_create(dipaco_ctx **out, int32_t num_levels, const int32_t *modules_p
  *   path_ptrs        HOST array [P] of DEVICE pointers, one per path copy; in/out
  *   reported         HOST [P], nonzero = path i reported; NULL = all reported
  *   cuda_stream      a cudaStream_t (0 = default stream)
- * With chunk_paths = 0 this is one fused pass; otherwise the library walks the chunks
- * (accumulate each chunk in ascending order, then write back) over the same device pointers.
+ * With chunk_paths = 0 this is one fused pass; otherwise the library walks the chunks in
+ * ascending order over the same device pointers, one launch per chunk, carrying fp32 partial
+ * sums; the launch that sees a module's last reporting path finishes the module and writes
+ * cast(theta') into all of its paths.  A call with the same settings, buffers and mask as the
+ * previous one on this context reuses that call's plan and device tables.
  */
 int dipaco_outer_sync(dipaco_ctx *ctx, float *theta, float *momentum, void *const *path_ptrs,
                       const uint8_t *reported, void *cuda_stream);
@@ -124,6 +127,9 @@ int dipaco_outer_sync(dipaco_ctx *ctx, float *theta, float *momentum, void *cons
  *              chunk's copies with cast(theta') (the contents of chunk_ptrs are not read, so the
  *              buffers may be fresh).
  *   end        checks that every chunk was accumulated and returns the context to idle.
+ * With bf16 copies the first begin on a context allocates a scratch of 2 bytes per module
+ * parameter: the finishing passes store cast(theta') there and the write-back launches read it
+ * instead of fp32 theta'.  If that allocation fails the write-back reads theta' (same results).
  */
 int dipaco_sync_begin(dipaco_ctx *ctx, float *theta, float *momentum, const uint8_t *reported,
                       void *cuda_stream);
@@ -208,6 +214,35 @@ int dipaco_set_input_kind(dipaco_ctx *ctx, int32_t input_kind);
  */
 int dipaco_set_shard(dipaco_ctx *ctx, int32_t shard_index, int32_t shard_count);
 
+/*
+ * The same partition for executors that hold ONLY their slab (Section 3.3: each executor of the
+ * sharded outer optimiser owns a part of the parameters and the matching part of every
+ * checkpoint).  Every module of level l has N_l elements, so shard s of S owns the same element
+ * range [begin_l, end_l) of every module of that level; dipaco_plan_shard returns it (host only,
+ * works on plan-only contexts).  Ranges are cut at multiples of 8192 elements, the last shard
+ * takes the remainder; over s = 0..S-1 they tile [0, N_l) exactly once.
+ */
+int dipaco_plan_shard(const dipaco_ctx *ctx, int32_t shard_index, int32_t shard_count, int32_t level,
+                      int64_t *begin, int64_t *end);
+
+/*
+ * A context for shard shard_index of shard_count of the problem that `whole` describes, in the
+ * compact layout: the shard is itself a module grid with the same levels, modules, paths and
+ * weights and with N_l replaced by end_l - begin_l.  Its theta, momentum (and second moment)
+ * hold, module after module, elements [begin_l, end_l) of each module; its path copies hold,
+ * level after level, elements [begin_l, end_l) of the path's slot: each executor allocates 1/S
+ * of everything and no pointer to the rest is ever needed.  Every entry point works on it as on
+ * any context, and the S results, put back side by side, are bit for bit the unsharded update:
+ * no exchange between executors (elements are independent).  The new context copies the
+ * weights, module scales, level flags, learning rate, momentum, optimiser, input kind, chunk
+ * size, kernel choice and tuning of `whole` as they are at the time of the call (`whole` may be
+ * plan-only and may be destroyed afterwards); the Adam family must be selected on the shard
+ * itself with dipaco_set_adam, because it needs the shard's own second-moment array.
+ * device: CUDA device of this executor, or -1 for plan only.
+ */
+int dipaco_create_shard(dipaco_ctx **out, const dipaco_ctx *whole, int32_t shard_index,
+                        int32_t shard_count, int32_t device);
+
 /* Choose the kernel family (DIPACO_KERNEL_*); all families give bitwise identical results. */
 int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
 
@@ -225,6 +260,15 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
                       int32_t units_per_thread, int32_t io_slots);
 
 /*
+ * Tuning of the bulk-copy kernel's dynamic scheduling: a launch is cut into work items (runs of
+ * tiles of one module) that the persistent CTAs draw from a counter.  An item moves at most
+ * max_item_bytes of traffic (default 2 MiB) and a launch is cut into at least items_per_cta
+ * items per CTA (default 16) so that the CTAs finish together.  0 keeps a value.  Results do not
+ * depend on the cut.
+ */
+int dipaco_set_work_items(dipaco_ctx *ctx, int64_t max_item_bytes, int32_t items_per_cta);
+
+/*
  * Tuning of dipaco_outer_sync_host: the most bytes of path data one streamed unit uploads
  * (0 = no cap other than the staging buffers).  Smaller units fill and drain the pipeline
  * faster, larger ones mean fewer and larger copies.
@@ -233,17 +277,35 @@ int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes);
 
 /*
  * Synchronise the context's last stream and report what the kernels recorded: DIPACO_OK, or
- * DIPACO_ETIMEOUT if a bounded wait gave up (results of that call are then undefined), or
- * DIPACO_ECUDA.  Clears the recorded status.
+ * DIPACO_ETIMEOUT if a bounded wait gave up, or DIPACO_ECUDA.  Clears the recorded status.
+ *
+ * Every wait inside the kernels is bounded (4 s).  A kernel whose wait runs out records a code
+ * in the context's error word and ends in an orderly way (copies in flight are waited for); the
+ * results of that call are undefined.  The error is sticky on the device: every later launch on
+ * the context sees the error word set and does nothing at all (buffers untouched, status of the
+ * entry point still DIPACO_OK since launches are asynchronous) until this function has been
+ * called; it returns DIPACO_ETIMEOUT once, re-arms the context (error word and work counters
+ * back to zero) and from then on calls work again.
  */
 int dipaco_device_status(dipaco_ctx *ctx);
+
+/*
+ * Diagnostic: make a bounded wait run out on purpose, harmlessly.  Launches one warp on the
+ * given stream whose first thread waits at most limit_ns (1 .. 1e9) on a barrier that nothing
+ * will complete; no copy is in flight and no buffer of the caller is involved.  When the wait
+ * gives up the kernel leaves what a pipeline kernel that gave up leaves: a code in the error
+ * word and a work counter that is not back at zero.  Afterwards the context behaves as after a
+ * real time-out (see dipaco_device_status).  Lets an application or a test check its handling of
+ * DIPACO_ETIMEOUT.  The paper has no counterpart.
+ */
+int dipaco_selftest_wait_expiry(dipaco_ctx *ctx, int64_t limit_ns, void *cuda_stream);
 
 /* Number of kernels this context has launched so far. */
 int64_t dipaco_launch_count(const dipaco_ctx *ctx);
 
 /*
- * Plan queries (host only; work on plan-only contexts too).  They expose step a0 of the path:
- * the contributor set of a module under a mask and the normalised coefficients.
+ * Plan queries (host only; work on plan-only contexts too).  They expose the host-side
+ * decisions: the contributor set of a module under a mask and the normalised coefficients.
  *   members / contributors  out, capacity num_paths each; ascending path ids
  *   coeff                   out, capacity num_paths; c_i as the kernels use them (fp32)
  *   will_update             out; 0 when no path reports or the total weight is zero
@@ -309,13 +371,19 @@ int dipaco_destroy(dipaco_ctx *ctx);
  *   device            CUDA device that owns all the buffers; made current during the call
  *   cuda_stream       stream the kernels are launched on (asynchronous)
  *
- * The static array: 16 MiB per GPU, held from the moment the library's CUDA module is loaded on
- * that GPU until the process exits, whether or not this function is ever called again.  The
- * first call on each device looks up the array's device address (cudaGetSymbolAddress); make
- * that first call before any stream capture begins.  All calls on one device share the array
- * and it keeps whatever the last call left in it: each call starts its sums from zero in the
- * kernel, so stale contents are never read, but two calls that overlap on the GPU (different
- * streams, or different host threads) race on it and must be serialised by the caller.
+ * The static array: 16 MiB per GPU.  It is part of the library's CUDA module, so the CUDA runtime
+ * reserves it when it loads that module on a GPU: with lazy module loading (the default) that is
+ * the first call of this function on the device, with eager loading the creation of the context.
+ * From then on the GPU holds the 16 MiB until the process exits, whether or not this function is
+ * called again.  The first call on a device (any numel >= 1) is therefore the set-up call: make
+ * it while the device still has room for the module (a caller that gives all device memory to
+ * its own pool makes it before that), and before any stream capture begins; if the module cannot
+ * be loaded it returns DIPACO_ENOMEM (or DIPACO_ECUDA), launches nothing and leaves no CUDA error
+ * pending.  Every call looks the array's device address up again (cudaGetSymbolAddress: no
+ * allocation once the module is loaded).  All calls on one device share the array and it keeps
+ * whatever the last call left in it: each call starts its sums from zero in the kernel, so stale
+ * contents are never read, but two calls that overlap on the GPU (different streams, or
+ * different host threads) race on it and must be serialised by the caller.
  */
 #define DIPACO_STATIC_MAX_NUMEL (4 * 1024 * 1024)
 int dipaco_module_sync_static(float *theta, float *momentum, int64_t numel, int32_t num_paths,

@@ -49,7 +49,8 @@ EXPORTS = [
     "dipaco_plan_chunks", "dipaco_plan_split", "dipaco_module_sync_static",
     "dipaco_set_host_unit_bytes", "dipaco_plan_traffic", "dipaco_set_module_scale",
     "dipaco_set_level_sync", "dipaco_set_shard", "dipaco_set_optimizer", "dipaco_set_adam",
-    "dipaco_set_input_kind",
+    "dipaco_set_input_kind", "dipaco_plan_shard", "dipaco_create_shard",
+    "dipaco_selftest_wait_expiry", "dipaco_set_work_items",
 ]
 
 _lib = None
@@ -86,11 +87,15 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_module_scale.argtypes = [vp, vp]
     lib.dipaco_set_level_sync.argtypes = [vp, vp]
     lib.dipaco_set_shard.argtypes = [vp, i32, i32]
+    lib.dipaco_plan_shard.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.dipaco_create_shard.argtypes = [ctypes.POINTER(vp), vp, i32, i32, i32]
+    lib.dipaco_selftest_wait_expiry.argtypes = [vp, i64, vp]
     lib.dipaco_set_optimizer.argtypes = [vp, i32]
     lib.dipaco_set_adam.argtypes = [vp, vp, f32, f32, f32, f32, i32]
     lib.dipaco_set_input_kind.argtypes = [vp, i32]
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32, i32]
+    lib.dipaco_set_work_items.argtypes = [vp, i64, i32]
     lib.dipaco_device_status.argtypes = [vp]
     lib.dipaco_set_host_unit_bytes.argtypes = [vp, i64]
     lib.dipaco_launch_count.argtypes = [vp]
@@ -122,8 +127,16 @@ def _np_ptr(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data
 
 
-def _ptr_array(ptrs: Sequence[int]):
+def _ptr_array(ptrs):
+    """A C array of pointers; one that ptr_array() already built is passed through."""
+    if isinstance(ptrs, ctypes.Array):
+        return ptrs
     return (ctypes.c_void_p * len(ptrs))(*[int(p) for p in ptrs])
+
+
+def ptr_array(ptrs: Sequence[int]):
+    """Build the C pointer array once, for callers that synchronise the same buffers repeatedly."""
+    return _ptr_array(ptrs)
 
 
 def _stream_handle(stream) -> int:
@@ -234,6 +247,27 @@ def dipaco_set_shard(ctx, shard_index: int, shard_count: int) -> None:
     _check(load().dipaco_set_shard(ctx, int(shard_index), int(shard_count)), "dipaco_set_shard")
 
 
+def dipaco_plan_shard(ctx, shard_index: int, shard_count: int, level: int):
+    """(begin, end): the element range of every module of `level` that the shard owns."""
+    a, b = ctypes.c_int64(), ctypes.c_int64()
+    _check(load().dipaco_plan_shard(ctx, int(shard_index), int(shard_count), int(level),
+                                    ctypes.addressof(a), ctypes.addressof(b)), "dipaco_plan_shard")
+    return a.value, b.value
+
+
+def dipaco_create_shard(whole: int, shard_index: int, shard_count: int, device=0) -> int:
+    """Context of one shard in the compact layout; returns its handle."""
+    handle = ctypes.c_void_p()
+    _check(load().dipaco_create_shard(ctypes.byref(handle), whole, int(shard_index), int(shard_count),
+                                      int(device)), "dipaco_create_shard")
+    return handle.value
+
+
+def dipaco_selftest_wait_expiry(ctx, limit_ns: int, stream=None) -> None:
+    _check(load().dipaco_selftest_wait_expiry(ctx, int(limit_ns), _stream_handle(stream)),
+           "dipaco_selftest_wait_expiry")
+
+
 def dipaco_set_kernel(ctx, kernel: int) -> None:
     _check(load().dipaco_set_kernel(ctx, int(kernel)), "dipaco_set_kernel")
 
@@ -241,6 +275,11 @@ def dipaco_set_kernel(ctx, kernel: int) -> None:
 def dipaco_set_tuning(ctx, ctas_per_sm=0, stages=0, units_per_thread=0, io_slots=0) -> None:
     _check(load().dipaco_set_tuning(ctx, int(ctas_per_sm), int(stages), int(units_per_thread),
                                     int(io_slots)), "dipaco_set_tuning")
+
+
+def dipaco_set_work_items(ctx, max_item_bytes=0, items_per_cta=0) -> None:
+    _check(load().dipaco_set_work_items(ctx, int(max_item_bytes), int(items_per_cta)),
+           "dipaco_set_work_items")
 
 
 def dipaco_set_host_unit_bytes(ctx, nbytes: int) -> None:

@@ -19,7 +19,6 @@ constexpr size_t SMEM_PER_SM = 228 * 1024;
 constexpr size_t SMEM_CTA_RESERVE = 1024;  // per-CTA reservation the driver adds
 constexpr int64_t RAGGED_TILE = 1024;      // split granularity of the scalar kernel
 constexpr int MAX_COUNTERS = 256;          // work counters (one per bulk launch of an upload)
-constexpr double ITEM_TARGET_BYTES = 2.0 * 1024 * 1024;  // traffic of one dynamic work item
 
 enum SyncState { STATE_IDLE = 0, STATE_ACCUMULATING = 1 };
 
@@ -62,6 +61,8 @@ struct dipaco_ctx {
     int kernel = DIPACO_KERNEL_AUTO;
     int ctas_per_sm = 1, stages = 10, units = 2;  // bulk-copy kernel tuning (measured on B200)
     int io_slots = 3;                            // buffers of theta/momentum/result tiles
+    int64_t item_bytes = 2 * 1024 * 1024;        // most traffic of one dynamic work item
+    int items_per_cta = 16;                      // least number of items per CTA that a launch is cut into
     int64_t launches = 0;
     int64_t host_unit_bytes = (int64_t)1 << 40;  // upload size cap of one unit in host mode
 
@@ -71,6 +72,8 @@ struct dipaco_ctx {
     int staging_next = 0;
     std::vector<unsigned char> last_blob;  // tables currently in dev_tables (skip identical uploads)
     float *partial = nullptr;
+    void *cast_scratch = nullptr;  // cast(theta') per module in the path dtype (chunk API, bf16 paths)
+    bool cast_scratch_tried = false;
     int *error_word = nullptr;
     int *counters = nullptr;  // MAX_COUNTERS work counters for the bulk-copy kernel
     bool smem_attr_set[2][3] = {{false, false, false}, {false, false, false}};
@@ -84,6 +87,13 @@ struct dipaco_ctx {
     int next_chunk = 0;
 
     HostMode *host_mode = nullptr;
+
+    // Plan of the last dipaco_outer_sync, kept while its tables are the ones on the device: a call
+    // with the same buffers, mask and settings launches again without planning or uploading.
+    uint64_t settings_version = 1;           // bumped by every dipaco_set_*
+    std::vector<unsigned char> plan_key;     // settings version, buffers, mask of the kept plan
+    std::vector<PackedLaunch> plan_launches;
+    bool plan_valid = false;
 };
 
 namespace {
@@ -101,6 +111,21 @@ struct DeviceGuard {
         if (prev >= 0) cudaSetDevice(prev);
     }
 };
+
+// Diagnostic kernel (dipaco_selftest_wait_expiry): one thread waits, with the given limit, on a
+// barrier phase that nothing will ever complete.  No copy is in flight and no other thread takes
+// part, so the only effect is what a pipeline CTA that gave up leaves behind: a code in the error
+// word and a work counter that is not back at zero.
+__global__ void wait_expiry_kernel(int *error_word, int *work_counter, unsigned long long limit_ns)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!bounded_wait(&bar, 0, error_word, 9, limit_ns)) atomicAdd(work_counter, 1);
+    }
+}
+
 
 void compute_all_coeffs(dipaco_ctx *ctx, const uint8_t *reported)
 {
@@ -176,6 +201,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         PassDev &pd = passes[i];
         pd.theta_off = m.theta_off;
         pd.partial_off = m.partial_off >= 0 ? m.partial_off : 0;
+        pd.cast_off = m.cast_off;
         pd.flags = sp.flags;
         pd.scale = sp.scale;
         pd.item_first = 0;
@@ -186,6 +212,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if ((sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) && (m.partial_off < 0 || !ctx->partial))
             return DIPACO_ESTATE;
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
+        if (((sp.flags & PASS_CAST_IN) || sp.cast_out) && !ctx->cast_scratch) return DIPACO_ESTATE;
         bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
                        ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
         if (ctx->optimizer == DIPACO_OPT_ADAM) {
@@ -212,6 +239,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
             aligned = aligned && ((uintptr_t)dst % 16 == 0);
             members.push_back(dst);
         }
+        if (sp.cast_out)  // the module's slot in the cast scratch is one more destination
+            members.push_back(static_cast<char *>(ctx->cast_scratch) + m.cast_off * es);
         if (extra_dst && i < extra_dst->size())
             for (void *dst : (*extra_dst)[i]) {
                 aligned = aligned && ((uintptr_t)dst % 16 == 0);
@@ -254,7 +283,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         split_segments(specs, bulk_begin, bulk_end, es, tile, bulk_ctas, bulk_segs, bulk_first);
     } else if (bulk_ctas > 0) {
         // Work items of about equal traffic, small enough that every CTA draws many of them.
-        const double target = std::min(ITEM_TARGET_BYTES, bulk_bytes / ((double)bulk_ctas * 16.0));
+        const double target =
+            std::min((double)ctx->item_bytes, bulk_bytes / ((double)bulk_ctas * (double)ctx->items_per_cta));
         for (size_t i = 0; i < specs.size(); ++i) {
             const int64_t ntiles = (bulk_end[i] - bulk_begin[i] + tile - 1) / tile;
             const double per_tile = pass_cost_per_elem(specs[i], es) * (double)tile;
@@ -306,6 +336,7 @@ int upload_blob(dipaco_ctx *ctx, const std::vector<unsigned char> &blob, cudaStr
         std::memcmp(blob.data(), ctx->last_blob.data(), blob.size()) == 0)
         return DIPACO_OK;  // same pointers, mask and weights as the previous call
     ctx->last_blob.clear();
+    ctx->plan_valid = false;  // the device tables are about to change
     if (bytes > ctx->dev_tables_capacity) {
         // grow: wait for earlier work that may still read the old tables
         if (cudaStreamSynchronize(stream) != cudaSuccess) return DIPACO_ECUDA;
@@ -394,6 +425,7 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
     lp.theta = theta;
     lp.momentum = momentum;
     lp.partial = ctx->partial;
+    lp.cast_scratch = ctx->cast_scratch;
     lp.passes = reinterpret_cast<const PassDev *>(base + pl.passes_off);
     lp.contribs = reinterpret_cast<const ContribDev *>(base + pl.contribs_off);
     lp.members = reinterpret_cast<void *const *>(base + pl.members_off);
@@ -453,8 +485,22 @@ struct LaunchRequest {
     std::vector<std::vector<void *>> extra_dst;
 };
 
+int launch_all(dipaco_ctx *ctx, const std::vector<PackedLaunch> &packed, float *theta, float *momentum,
+               cudaStream_t stream)
+{
+    for (size_t i = 0; i < packed.size(); ++i) {
+        // every bulk launch leaves its pair of counters at zero again, so pairs can be reused
+        // by later launches on the same stream
+        const int c = (int)(i % MAX_COUNTERS);
+        const int rc = launch_packed(ctx, packed[i], theta, momentum, ctx->counters + 2 * c, stream);
+        if (rc != DIPACO_OK) return rc;
+    }
+    ctx->last_stream = stream;
+    return DIPACO_OK;
+}
+
 int run_launches(dipaco_ctx *ctx, std::vector<LaunchRequest> &reqs, float *theta, float *momentum,
-                 cudaStream_t stream)
+                 cudaStream_t stream, std::vector<PackedLaunch> *keep = nullptr)
 {
     std::vector<unsigned char> blob;
     std::vector<PackedLaunch> packed(reqs.size());
@@ -466,15 +512,9 @@ int run_launches(dipaco_ctx *ctx, std::vector<LaunchRequest> &reqs, float *theta
     }
     int rc = upload_blob(ctx, blob, stream);
     if (rc != DIPACO_OK) return rc;
-    for (size_t i = 0; i < reqs.size(); ++i) {
-        // every bulk launch leaves its pair of counters at zero again, so pairs can be reused
-        // by later launches on the same stream
-        const int c = (int)(i % MAX_COUNTERS);
-        rc = launch_packed(ctx, packed[i], theta, momentum, ctx->counters + 2 * c, stream);
-        if (rc != DIPACO_OK) return rc;
-    }
-    ctx->last_stream = stream;
-    return DIPACO_OK;
+    rc = launch_all(ctx, packed, theta, momentum, stream);
+    if (rc == DIPACO_OK && keep) *keep = std::move(packed);
+    return rc;
 }
 
 bool valid_ptr_array(void *const *ptrs, int n)
@@ -570,6 +610,7 @@ int dipaco_destroy(dipaco_ctx *ctx)
         }
         if (ctx->dev_tables) cudaFree(ctx->dev_tables);
         if (ctx->partial) cudaFree(ctx->partial);
+        if (ctx->cast_scratch) cudaFree(ctx->cast_scratch);
         if (ctx->error_word) cudaFree(ctx->error_word);
         if (ctx->counters) cudaFree(ctx->counters);
     }
@@ -581,6 +622,7 @@ int dipaco_set_weights(dipaco_ctx *ctx, const float *path_weights)
 {
     if (!ctx) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     if (path_weights) {
         for (int i = 0; i < ctx->grid.P; ++i)
             if (!(path_weights[i] >= 0.0f) || !std::isfinite(path_weights[i])) return DIPACO_EINVAL;
@@ -595,6 +637,7 @@ int dipaco_set_module_scale(dipaco_ctx *ctx, const float *module_scale)
 {
     if (!ctx) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     if (module_scale) {
         const size_t n = ctx->grid.modules.size();
         for (size_t i = 0; i < n; ++i)
@@ -610,6 +653,7 @@ int dipaco_set_level_sync(dipaco_ctx *ctx, const uint8_t *level_sync)
 {
     if (!ctx) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     if (level_sync) ctx->grid.level_sync.assign(level_sync, level_sync + ctx->grid.L);
     else ctx->grid.level_sync.clear();
     return DIPACO_OK;
@@ -619,6 +663,7 @@ int dipaco_set_optimizer(dipaco_ctx *ctx, int32_t optimizer)
 {
     if (!ctx || optimizer < DIPACO_OPT_NESTEROV || optimizer > DIPACO_OPT_ADAM) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     if (optimizer == DIPACO_OPT_ADAM && !ctx->second_moment) return DIPACO_ESTATE;  // dipaco_set_adam first
     ctx->optimizer = optimizer;
     ctx->grid.second_moment = optimizer == DIPACO_OPT_ADAM;
@@ -632,6 +677,7 @@ int dipaco_set_adam(dipaco_ctx *ctx, float *second_moment, float beta1, float be
     if (!(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f)) return DIPACO_EINVAL;
     if (!(eps >= 0.0f) || !std::isfinite(eps) || !std::isfinite(weight_decay)) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     ctx->second_moment = second_moment;
     ctx->adam_b1 = beta1;
     ctx->adam_b2 = beta2;
@@ -648,6 +694,7 @@ int dipaco_set_input_kind(dipaco_ctx *ctx, int32_t input_kind)
     if (!ctx || (input_kind != DIPACO_INPUT_COPIES && input_kind != DIPACO_INPUT_GRADIENTS))
         return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     ctx->input_kind = input_kind;
     return DIPACO_OK;
 }
@@ -656,6 +703,7 @@ int dipaco_set_shard(dipaco_ctx *ctx, int32_t shard_index, int32_t shard_count)
 {
     if (!ctx || shard_count < 1 || shard_index < 0 || shard_index >= shard_count) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     ctx->grid.shard_index = shard_index;
     ctx->grid.shard_count = shard_count;
     return DIPACO_OK;
@@ -665,6 +713,7 @@ int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel)
 {
     if (!ctx || kernel < DIPACO_KERNEL_AUTO || kernel > DIPACO_KERNEL_SCALAR) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     ctx->kernel = kernel;
     return DIPACO_OK;
 }
@@ -674,6 +723,7 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
 {
     if (!ctx) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     if (ctas_per_sm < 0 || ctas_per_sm > 8 || stages < 0 || stages == 1 || stages > BULK_MAX_STAGES)
         return DIPACO_EINVAL;
     if (units_per_thread != 0 && units_per_thread != 1 && units_per_thread != 2 && units_per_thread != 4)
@@ -697,10 +747,21 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
     return DIPACO_OK;
 }
 
+int dipaco_set_work_items(dipaco_ctx *ctx, int64_t max_item_bytes, int32_t items_per_cta)
+{
+    if (!ctx || max_item_bytes < 0 || items_per_cta < 0 || items_per_cta > 4096) return DIPACO_EINVAL;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
+    if (max_item_bytes) ctx->item_bytes = max_item_bytes;
+    if (items_per_cta) ctx->items_per_cta = items_per_cta;
+    return DIPACO_OK;
+}
+
 int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes)
 {
     if (!ctx || bytes < 0) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    ++ctx->settings_version;
     ctx->host_unit_bytes = bytes == 0 ? (int64_t)1 << 40 : bytes;
     return DIPACO_OK;
 }
@@ -716,6 +777,18 @@ int dipaco_sync_begin(dipaco_ctx *ctx, float *theta, float *momentum, const uint
         compute_all_coeffs(ctx, reported);
     } catch (const std::bad_alloc &) {
         return DIPACO_ENOMEM;
+    }
+    // bf16 copies: the write-back launches of this API read cast(theta') (2 bytes per parameter)
+    // from a scratch that the finishing passes fill, instead of fp32 theta'.  Allocated on the
+    // first round; without it (no memory) the write-back reads theta' as before.
+    if (ctx->elem_size != 4 && !ctx->cast_scratch && !ctx->cast_scratch_tried && ctx->grid.cast_elems > 0) {
+        ctx->cast_scratch_tried = true;
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok) return DIPACO_ECUDA;
+        if (cudaMalloc(&ctx->cast_scratch, (size_t)ctx->grid.cast_elems * ctx->elem_size) != cudaSuccess) {
+            cudaGetLastError();
+            ctx->cast_scratch = nullptr;
+        }
     }
     ctx->theta = theta;
     ctx->momentum = momentum;
@@ -737,7 +810,8 @@ int dipaco_sync_accumulate(dipaco_ctx *ctx, int32_t chunk_index, void *const *ch
     if (!guard.ok) return DIPACO_ECUDA;
     try {
         std::vector<LaunchRequest> reqs(1);
-        plan_accumulate(ctx->grid, ctx->coeffs, chunk_index, reqs[0].specs);
+        plan_accumulate(ctx->grid, ctx->coeffs, chunk_index, reqs[0].specs, false,
+                        ctx->cast_scratch != nullptr);
         reqs[0].lookup = PtrLookup{chunk_ptrs, chunk_first(ctx->grid, chunk_index), n};
         if (!reqs[0].specs.empty()) {
             const int rc = run_launches(ctx, reqs, ctx->theta, ctx->momentum, ctx->stream);
@@ -762,7 +836,8 @@ int dipaco_sync_writeback(dipaco_ctx *ctx, int32_t chunk_index, void *const *chu
     if (!guard.ok) return DIPACO_ECUDA;
     try {
         std::vector<LaunchRequest> reqs(1);
-        plan_writeback(ctx->grid, ctx->coeffs, chunk_index, false, reqs[0].specs);
+        plan_writeback(ctx->grid, ctx->coeffs, chunk_index, false, reqs[0].specs,
+                       ctx->cast_scratch != nullptr);
         reqs[0].lookup = PtrLookup{chunk_ptrs, chunk_first(ctx->grid, chunk_index), n};
         if (!reqs[0].specs.empty()) {
             const int rc = run_launches(ctx, reqs, ctx->theta, ctx->momentum, ctx->stream);
@@ -796,31 +871,60 @@ int dipaco_outer_sync(dipaco_ctx *ctx, float *theta, float *momentum, void *cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const Grid &g = ctx->grid;
     try {
+        // Same settings, buffers and mask as the previous call, and its tables are still the ones
+        // on the device: launch again, nothing to plan or upload.
+        const size_t P = (size_t)g.P;
+        std::vector<unsigned char> key(sizeof(uint64_t) + 3 * sizeof(void *) + 1 + P + P * sizeof(void *));
+        {
+            unsigned char *k = key.data();
+            const void *fixed[3] = {theta, momentum, ctx->second_moment};
+            std::memcpy(k, &ctx->settings_version, sizeof(uint64_t)); k += sizeof(uint64_t);
+            std::memcpy(k, fixed, sizeof fixed); k += sizeof fixed;
+            *k++ = reported ? 1 : 0;
+            if (reported) for (size_t i = 0; i < P; ++i) k[i] = reported[i] ? 1 : 0;
+            else std::memset(k, 1, P);
+            k += P;
+            std::memcpy(k, path_ptrs, P * sizeof(void *));
+        }
+        if (ctx->plan_valid && key == ctx->plan_key)
+            return launch_all(ctx, ctx->plan_launches, theta, momentum, stream);
+        ctx->plan_valid = false;
+
         compute_all_coeffs(ctx, reported);
         std::vector<LaunchRequest> reqs;
+        const PtrLookup all_paths{path_ptrs, 0, g.P};
         if (g.num_chunks <= 1) {
             reqs.resize(1);
             plan_resident(g, ctx->coeffs, reqs[0].specs);
-            reqs[0].lookup = PtrLookup{path_ptrs, 0, g.P};
+            reqs[0].lookup = all_paths;
         } else {
-            // accumulate every chunk in ascending order, then fill the slots that were not final yet
+            // Walk the chunks in ascending order.  Every path copy is on the device here, so the
+            // pass that finishes a module hands cast(theta') to all its paths at once, whatever
+            // their chunk; modules that nobody updates are refilled in the first launch.
             for (int c = 0; c < g.num_chunks; ++c) {
                 LaunchRequest r;
-                plan_accumulate(g, ctx->coeffs, c, r.specs);
-                r.lookup = PtrLookup{path_ptrs + chunk_first(g, c), chunk_first(g, c), chunk_count(g, c)};
+                plan_accumulate(g, ctx->coeffs, c, r.specs, true);
+                r.lookup = all_paths;
                 if (!r.specs.empty()) reqs.push_back(std::move(r));
             }
-            for (int c = 0; c < g.num_chunks; ++c) {
-                LaunchRequest r;
-                plan_writeback(g, ctx->coeffs, c, true, r.specs);
-                r.lookup = PtrLookup{path_ptrs + chunk_first(g, c), chunk_first(g, c), chunk_count(g, c)};
-                if (!r.specs.empty()) reqs.push_back(std::move(r));
+            LaunchRequest refill;
+            plan_refill_unchanged(g, ctx->coeffs, refill.specs);
+            refill.lookup = all_paths;
+            if (!refill.specs.empty()) {
+                if (reqs.empty()) reqs.push_back(std::move(refill));
+                else
+                    for (PassSpec &sp : refill.specs) reqs[0].specs.push_back(std::move(sp));
             }
         }
         bool any = false;
         for (auto &r : reqs) any = any || !r.specs.empty();
         if (!any) return DIPACO_OK;
-        return run_launches(ctx, reqs, theta, momentum, stream);
+        const int rc = run_launches(ctx, reqs, theta, momentum, stream, &ctx->plan_launches);
+        if (rc == DIPACO_OK) {
+            ctx->plan_key = std::move(key);
+            ctx->plan_valid = true;
+        }
+        return rc;
     } catch (const std::bad_alloc &) {
         return DIPACO_ENOMEM;
     }
@@ -842,6 +946,75 @@ int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_h
     } catch (const std::bad_alloc &) {
         return DIPACO_ENOMEM;
     }
+}
+
+int dipaco_plan_shard(const dipaco_ctx *ctx, int32_t shard_index, int32_t shard_count, int32_t level,
+                      int64_t *begin, int64_t *end)
+{
+    if (!ctx || shard_count < 1 || shard_index < 0 || shard_index >= shard_count || level < 0 ||
+        level >= ctx->grid.L)
+        return DIPACO_EINVAL;
+    int64_t lo = 0, hi = 0;
+    Grid::slab_bounds(ctx->grid.N[(size_t)level], shard_index, shard_count, lo, hi);
+    if (begin) *begin = lo;
+    if (end) *end = hi;
+    return DIPACO_OK;
+}
+
+int dipaco_create_shard(dipaco_ctx **out, const dipaco_ctx *whole, int32_t shard_index,
+                        int32_t shard_count, int32_t device)
+{
+    if (!out) return DIPACO_EINVAL;
+    *out = nullptr;
+    if (!whole || shard_count < 1 || shard_index < 0 || shard_index >= shard_count) return DIPACO_EINVAL;
+    const Grid &g = whole->grid;
+    if (g.shard_count != 1) return DIPACO_ESTATE;  // a shard of a shard is not defined
+    try {
+        std::vector<int64_t> slab((size_t)g.L);
+        for (int l = 0; l < g.L; ++l) {
+            int64_t lo = 0, hi = 0;
+            Grid::slab_bounds(g.N[(size_t)l], shard_index, shard_count, lo, hi);
+            slab[(size_t)l] = hi - lo;
+        }
+        std::vector<int32_t> K(g.K.begin(), g.K.end()), table(g.table.begin(), g.table.end());
+        dipaco_ctx *ctx = nullptr;
+        const int rc = dipaco_create(&ctx, g.L, K.data(), slab.data(), g.P, table.data(),
+                                     g.weights.empty() ? nullptr : g.weights.data(), whole->lr, whole->mu,
+                                     whole->dtype, g.chunk_paths, device);
+        if (rc != DIPACO_OK) return rc;
+        ctx->grid.module_scale = g.module_scale;
+        ctx->grid.level_sync = g.level_sync;
+        ctx->input_kind = whole->input_kind;
+        ctx->kernel = whole->kernel;
+        ctx->ctas_per_sm = whole->ctas_per_sm;
+        ctx->stages = whole->stages;
+        ctx->units = whole->units;
+        ctx->io_slots = whole->io_slots;
+        ctx->item_bytes = whole->item_bytes;
+        ctx->items_per_cta = whole->items_per_cta;
+        ctx->host_unit_bytes = whole->host_unit_bytes;
+        // the Adam family needs the shard's own second-moment array: dipaco_set_adam on the shard
+        ctx->optimizer = whole->optimizer == DIPACO_OPT_ADAM ? DIPACO_OPT_NESTEROV : whole->optimizer;
+        *out = ctx;
+        return DIPACO_OK;
+    } catch (const std::bad_alloc &) {
+        return DIPACO_ENOMEM;
+    }
+}
+
+int dipaco_selftest_wait_expiry(dipaco_ctx *ctx, int64_t limit_ns, void *cuda_stream)
+{
+    if (!ctx || limit_ns < 1 || limit_ns > 1000000000ll) return DIPACO_EINVAL;
+    if (ctx->device < 0) return DIPACO_ENODEV;
+    if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DIPACO_ECUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    wait_expiry_kernel<<<1, 32, 0, stream>>>(ctx->error_word, ctx->counters,
+                                             (unsigned long long)limit_ns);
+    if (cudaGetLastError() != cudaSuccess) return DIPACO_ECUDA;
+    ctx->last_stream = stream;
+    return DIPACO_OK;
 }
 
 int dipaco_device_status(dipaco_ctx *ctx)
@@ -929,8 +1102,19 @@ int dipaco_plan_traffic(const dipaco_ctx *ctx, const uint8_t *reported, int64_t 
             plan_resident(g, mc, specs);
             add();
         } else {
-            for (int c = 0; c < g.num_chunks; ++c) { plan_accumulate(g, mc, c, specs); add(); }
-            for (int c = 0; c < g.num_chunks; ++c) { plan_writeback(g, mc, c, true, specs); add(); }
+            // as dipaco_outer_sync walks them: the refill passes ride in the first launch
+            std::vector<PassSpec> refill;
+            plan_refill_unchanged(g, mc, refill);
+            bool first = true;
+            for (int c = 0; c < g.num_chunks; ++c) {
+                plan_accumulate(g, mc, c, specs, true);
+                if (specs.empty()) continue;
+                if (first)
+                    for (PassSpec &sp : refill) specs.push_back(sp);
+                first = false;
+                add();
+            }
+            if (first) { specs = refill; add(); }
         }
         if (bytes) *bytes = (int64_t)total;
         if (launches) *launches = count;

@@ -11,6 +11,9 @@
 //     D2H  theta'[a:b], m'[a:b], and the output buffer into the slot of every path of the module
 // Units are double-buffered over three streams, so the upload of unit n+1, the kernel of unit n
 // and the download of unit n-1 overlap; a step costs about max(H2D bytes, D2H bytes) / PCIe rate.
+// The first units are small and double in size up to the steady size, and the last ones halve
+// again, so that the time before the first kernel (nothing overlaps the first upload) and after the
+// last one (nothing overlaps the last download) stays in the millisecond range.
 // The staging memory is bounded by chunk_paths path copies.  Paths that did not report are never
 // uploaded.  Bitwise identical to the resident mode: same pass, same order.
 
@@ -100,6 +103,77 @@ int host_mode_prepare(dipaco_ctx *ctx)
     return DIPACO_OK;
 }
 
+// One streamed unit: elements [a, b) of one module.
+struct HostUnit {
+    int module;
+    int64_t a, b;
+};
+
+constexpr size_t HOST_RAMP_BASE = (size_t)16 << 20;  // bytes one direction moves in the first / last unit
+
+// Cut the round into units.  Steady size: every reporting copy's piece fits one input buffer, the
+// cast piece fits the output buffer, and the upload stays under the configured cap.  Unit k from
+// the start and unit k from the end move at most HOST_RAMP_BASE * 2^k bytes in either direction.
+int plan_host_units(const dipaco_ctx *ctx, const HostMode *h, std::vector<HostUnit> &units)
+{
+    const Grid &g = ctx->grid;
+    const int es = ctx->elem_size;
+    const int64_t tile = tile_elems(ctx);
+    units.clear();
+    auto bytes_per_elem = [&](size_t id) -> size_t {
+        const size_t up = ctx->coeffs[id].contributors.size(), down = g.modules[id].members.size();
+        return std::max(up, down) * (size_t)es + 2 * sizeof(float);
+    };
+    auto ramp_elems = [&](size_t id, size_t k) -> int64_t {
+        const size_t cap = HOST_RAMP_BASE << std::min<size_t>(k, 24);
+        return std::max<int64_t>(tile, (int64_t)(cap / bytes_per_elem(id)) / tile * tile);
+    };
+    for (size_t id = 0; id < g.modules.size(); ++id) {
+        const ModuleGeom &m = g.modules[id];
+        const ModuleCoeffs &mc = ctx->coeffs[id];
+        if (m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
+        const size_t ncon = mc.contributors.size();
+        const size_t in_budget = std::max<size_t>(std::min(h->stage_in_bytes, (size_t)ctx->host_unit_bytes),
+                                                  ncon * (size_t)tile * es);
+        int64_t slab = m.numel;
+        if (ncon > 0 && ncon * align_up((size_t)m.numel * es, 256) > in_budget) {
+            const int64_t fit = (int64_t)(in_budget / (ncon * (size_t)es));
+            slab = fit / tile * tile;  // a tile's bytes are a multiple of the 256-byte piece stride
+        }
+        if ((size_t)slab * es > h->stage_out_bytes)
+            slab = (int64_t)(h->stage_out_bytes / (size_t)es) / tile * tile;
+        if (slab < 1) return DIPACO_ENOMEM;
+        int64_t lo = 0, hi = m.numel;
+        g.shard_range(m, lo, hi);
+        for (int64_t a = lo; a < hi;) {
+            const int64_t n = std::min(slab, ramp_elems(id, units.size()));
+            const int64_t b = std::min(hi, a + n);
+            units.push_back(HostUnit{(int)id, a, b});
+            a = b;
+        }
+    }
+    // the same ramp from the end: split the last units until unit k from the end fits its cap
+    std::vector<HostUnit> tail;
+    while (!units.empty() && tail.size() < 24) {
+        HostUnit &u = units.back();
+        const int64_t cap = ramp_elems((size_t)u.module, tail.size());
+        if (u.b - u.a > cap) {
+            const int64_t cut = (u.b - cap) / tile * tile;  // unit starts stay on tile boundaries
+            if (cut > u.a) {
+                tail.push_back(HostUnit{u.module, cut, u.b});
+                u.b = cut;
+                continue;
+            }
+        }
+        const bool steady = (size_t)cap * bytes_per_elem((size_t)u.module) >= h->stage_in_bytes;
+        tail.push_back(u);
+        units.pop_back();
+        if (steady) break;
+    }
+    units.insert(units.end(), tail.rbegin(), tail.rend());
+    return DIPACO_OK;
+}
+
 int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
                    void *const *path_ptrs_host, const uint8_t *reported, cudaStream_t stream)
 {
@@ -124,6 +198,20 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
         ~StagedSecondMoment() { c->second_moment_staged = nullptr; }
     } staged(ctx, adam ? h->second_d : nullptr);
 
+    // Whatever way this function is left, no copy may still be running into (or out of) the
+    // caller's host buffers: the call is synchronous, and after an error the caller is free to
+    // release them at once.
+    struct DrainOnExit {
+        HostMode *h;
+        cudaStream_t main;
+        ~DrainOnExit()
+        {
+            cudaStreamSynchronize(h->in_stream);
+            cudaStreamSynchronize(main);
+            cudaStreamSynchronize(h->out_stream);
+        }
+    } drain{h, stream};
+
     // the side streams must not run ahead of work queued earlier on the caller's stream
     if (cudaEventRecord(h->main_ready, stream) != cudaSuccess ||
         cudaStreamWaitEvent(h->in_stream, h->main_ready, 0) != cudaSuccess ||
@@ -131,28 +219,17 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
         return DIPACO_ECUDA;
 
     std::vector<void *> by_path((size_t)g.P, nullptr);
+    std::vector<HostUnit> units;
+    rc = plan_host_units(ctx, h, units);
+    if (rc != DIPACO_OK) return rc;
     long long unit_index = 0;
-    for (size_t id = 0; id < g.modules.size(); ++id) {
-        const ModuleGeom &m = g.modules[id];
-        const ModuleCoeffs &mc = ctx->coeffs[id];
-        if (m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
-        const size_t ncon = mc.contributors.size();
-        // elements per unit: every reporting copy's piece must fit the input buffer
-        // and a unit uploads at most HOST_UNIT_BYTES so that the pipeline fills and drains quickly
-        const size_t in_budget = std::max<size_t>(std::min(h->stage_in_bytes, (size_t)ctx->host_unit_bytes),
-                                                  ncon * (size_t)tile * es);
-        int64_t slab = m.numel;
-        if (ncon > 0 && ncon * align_up((size_t)m.numel * es, 256) > in_budget) {
-            const int64_t fit = (int64_t)(in_budget / (ncon * (size_t)es));
-            slab = fit / tile * tile;  // a tile's bytes are a multiple of the 256-byte piece stride
-        }
-        if ((size_t)slab * es > h->stage_out_bytes)
-            slab = (int64_t)(h->stage_out_bytes / (size_t)es) / tile * tile;
-        if (slab < 1) return DIPACO_ENOMEM;
-        int64_t shard_lo = 0, shard_hi = m.numel;
-        g.shard_range(m, shard_lo, shard_hi);
-        for (int64_t a = shard_lo; a < shard_hi; a += slab, ++unit_index) {
-            const int64_t b = std::min<int64_t>(shard_hi, a + slab);
+    for (const HostUnit &unit : units) {
+        {
+            const size_t id = (size_t)unit.module;
+            const ModuleGeom &m = g.modules[id];
+            const ModuleCoeffs &mc = ctx->coeffs[id];
+            const size_t ncon = mc.contributors.size();
+            const int64_t a = unit.a, b = unit.b;
             const int buf = (int)(unit_index & 1);
             const size_t piece = (size_t)(b - a) * es;
             const size_t piece_stride = align_up(piece, 256);
@@ -233,6 +310,7 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
                     return DIPACO_ECUDA;
             }
             if (cudaEventRecord(h->out_done[buf], h->out_stream) != cudaSuccess) return DIPACO_ECUDA;
+            ++unit_index;
         }
     }
     if (cudaStreamSynchronize(h->in_stream) != cudaSuccess ||

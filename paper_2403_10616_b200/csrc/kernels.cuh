@@ -17,11 +17,18 @@
 
 namespace dipaco {
 
-enum : int { KPASS_UPDATE = 1, KPASS_PARTIAL_IN = 2, KPASS_PARTIAL_OUT = 4 };
+enum : int {
+    KPASS_UPDATE = 1,
+    KPASS_PARTIAL_IN = 2,
+    KPASS_PARTIAL_OUT = 4,
+    KPASS_CAST_IN = 8,  // write-back only pass: cast(theta') is read from the cast scratch (path
+                        // dtype) instead of being derived from fp32 theta'
+};
 
 struct PassDev {
     long long theta_off;    // elements into theta / momentum
     long long partial_off;  // elements into the partial-sum scratch (valid with PARTIAL flags)
+    long long cast_off;     // elements into the cast scratch (valid with KPASS_CAST_IN)
     int contrib_begin, contrib_count;
     int member_begin, member_count;
     int flags;
@@ -63,6 +70,7 @@ struct LaunchParams {
     float *theta;
     float *momentum;
     float *partial;
+    const void *cast_scratch;  // cast(theta') of finished modules in the path dtype (chunk API)
     const PassDev *passes;
     const ContribDev *contribs;
     void *const *members;  // start of the module's slot inside each member path copy
@@ -183,6 +191,9 @@ template <> struct Unit<__nv_bfloat16> {
 template <typename PathT, int VEC>
 __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
 {
+    // a context whose error word is set (a bounded wait ran out earlier) does no further work
+    // until the host has read the status
+    if (*reinterpret_cast<volatile const int *>(p.error_word) != 0) return;
     const int seg_begin = p.cta_first[blockIdx.x];
     const int seg_end = p.cta_first[blockIdx.x + 1];
     for (int s = seg_begin; s < seg_end; ++s) {
@@ -193,12 +204,14 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
         float *theta = p.theta + pass.theta_off;
         float *momentum = p.momentum + pass.theta_off;
         float *partial = p.partial + pass.partial_off;
+        const PathT *cast_src = static_cast<const PathT *>(p.cast_scratch) + pass.cast_off;
 
         for (long long k = seg.begin + (long long)threadIdx.x * VEC; k < seg.end;
              k += (long long)blockDim.x * VEC) {
             float th[VEC], acc[VEC];
             if constexpr (VEC == 1) {
-                th[0] = theta[k];
+                // widening the stored cast and narrowing it again reproduces its bits exactly
+                th[0] = (pass.flags & KPASS_CAST_IN) ? PathIO<PathT>::load(cast_src + k) : theta[k];
                 acc[0] = (pass.flags & KPASS_PARTIAL_IN) ? partial[k] : 0.0f;
                 // loads of four contributors in flight, summation still in ascending order
                 int j = 0;
@@ -222,10 +235,16 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
                 constexpr int UE = Unit<PathT>::UE;
                 constexpr int UNITS = VEC / UE;  // 16-byte loads per contributor
                 constexpr int BATCH = 8 / UNITS; // contributors whose loads are issued together
+                if (pass.flags & KPASS_CAST_IN) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(cast_src + k);
 #pragma unroll
-                for (int v = 0; v < VEC; v += 4) {
-                    const float4 t = *reinterpret_cast<const float4 *>(theta + k + v);
-                    th[v] = t.x; th[v + 1] = t.y; th[v + 2] = t.z; th[v + 3] = t.w;
+                    for (int u = 0; u < UNITS; ++u) Unit<PathT>::widen(__ldcs(src + u), th + u * UE);
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VEC; v += 4) {
+                        const float4 t = *reinterpret_cast<const float4 *>(theta + k + v);
+                        th[v] = t.x; th[v + 1] = t.y; th[v + 2] = t.z; th[v + 3] = t.w;
+                    }
                 }
                 if (pass.flags & KPASS_PARTIAL_IN) {
 #pragma unroll
@@ -420,7 +439,8 @@ constexpr int BULK_ITEM_READERS = BULK_COMPUTE_WARPS + 2;  // warps that consume
 constexpr unsigned long long BULK_WAIT_LIMIT_NS = 4000000000ull;  // every wait gives up after 4 s
 
 // Bounded wait: returns false (and records the failure) if the phase does not complete in time.
-__device__ __forceinline__ bool bounded_wait(uint64_t *bar, unsigned parity, int *error_word, int code)
+__device__ __forceinline__ bool bounded_wait(uint64_t *bar, unsigned parity, int *error_word, int code,
+                                             unsigned long long limit_ns = BULK_WAIT_LIMIT_NS)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = ptx::global_timer_ns();
@@ -428,7 +448,7 @@ __device__ __forceinline__ bool bounded_wait(uint64_t *bar, unsigned parity, int
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (ptx::mbar_try_wait(bar, parity)) return true;
-        if (ptx::global_timer_ns() - t0 > BULK_WAIT_LIMIT_NS) {
+        if (ptx::global_timer_ns() - t0 > limit_ns) {
             atomicCAS(error_word, 0, code);
             return false;
         }
@@ -573,8 +593,19 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
         if (lane == 0) {
             int slot = 0;
             unsigned phase = 0;
+            // A context whose error word is already set (a bounded wait ran out in an earlier
+            // launch) does no further work until the host has read the status: this CTA publishes
+            // its end-of-work marker at once and leaves the work counters alone.
+            const bool poisoned = *reinterpret_cast<volatile const int *>(p.error_word) != 0;
             for (;;) {
                 if (!bounded_wait(&sh->sched_empty[slot], phase ^ 1u, p.error_word, 8)) break;
+                if (poisoned) {
+                    sh->sched_pass[slot] = -1;
+                    sh->sched_begin[slot] = 0;
+                    sh->sched_end[slot] = 0;
+                    ptx::mbar_arrive(&sh->sched_full[slot]);
+                    break;
+                }
                 const int item = atomicAdd(p.work_counter, 1);
                 int item_pass = -1;
                 long long b = 0, e = 0;
@@ -615,7 +646,14 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
             const int b = io_pos.slot;
             if (lane == 0) {
                 ok = bounded_wait(&sh->io_empty[b], io_pos.phase ^ 1u, p.error_word, 1);
-                if (ok) {
+                if (ok && (pass.flags & KPASS_CAST_IN)) {
+                    // write-back only: the finished cast tile comes straight from the scratch
+                    const unsigned path_bytes = n * (unsigned)sizeof(PathT);
+                    ptx::mbar_arrive_expect_tx(&sh->io_full[b], path_bytes);
+                    ptx::bulk_load(cast_tile(b),
+                                   static_cast<const PathT *>(p.cast_scratch) + pass.cast_off + k0,
+                                   path_bytes, &sh->io_full[b]);
+                } else if (ok) {
                     const unsigned f32_bytes = n * 4u;
                     unsigned bytes = f32_bytes;
                     const bool adam = (pass.flags & KPASS_UPDATE) && p.rule.optimizer == KOPT_ADAM;
@@ -716,6 +754,13 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
             const int b = io_pos.slot;
             ok = bounded_wait(&sh->io_full[b], io_pos.phase, p.error_word, 5);
             if (!ok) break;
+            if (pass.flags & KPASS_CAST_IN) {
+                // the cast tile arrived ready-made: hand it on to the store warp
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&sh->out_ready[b]);
+                io_pos.advance(io_slots);
+                continue;
+            }
             float th[EPT], acc[EPT];
             float *th_tile = io_tile(b, 0);
 #pragma unroll

@@ -15,6 +15,7 @@ enum : int {
     PASS_UPDATE = 1,       // apply the Nesterov step and store theta', m'
     PASS_PARTIAL_IN = 2,   // start the reduction from the stored partial sum
     PASS_PARTIAL_OUT = 4,  // store the running sum instead of updating
+    PASS_CAST_IN = 8,      // write-back only: read cast(theta') from the cast scratch, not fp32 theta'
 };
 
 struct ModuleGeom {
@@ -23,6 +24,7 @@ struct ModuleGeom {
     int64_t path_off = 0;     // elements into a path copy (start of the level)
     int64_t numel = 0;
     int64_t partial_off = -1; // elements into the partial-sum scratch, -1 = none
+    int64_t cast_off = 0;     // elements into the cast scratch (every module has a slot)
     std::vector<int> members; // ascending path ids through this module  (S(l,e))
 };
 
@@ -39,6 +41,7 @@ struct Grid {
     int64_t module_params = 0, params_per_path = 0;
     int chunk_paths = 0, num_chunks = 1;
     int64_t scratch_elems = 0;
+    int64_t cast_elems = 0;                // size of the cast scratch in path elements
     int shard_index = 0, shard_count = 1;  // this context owns one slab of every module
     bool second_moment = false;            // the optimiser keeps a second state array (Adam family)
 
@@ -49,15 +52,21 @@ struct Grid {
     // elements (a multiple of every tile size), the last shard takes the remainder.
     void shard_range(const ModuleGeom &m, int64_t &lo, int64_t &hi) const
     {
+        slab_bounds(m.numel, shard_index, shard_count, lo, hi);
+    }
+    // Slab `index` of `count` of a module of `numel` elements.  Every module of a level has the
+    // same size, so the bounds are a property of the level.
+    static void slab_bounds(int64_t numel, int index, int count, int64_t &lo, int64_t &hi)
+    {
         const int64_t grain = 8192;
         auto cut = [&](int i) -> int64_t {
             if (i <= 0) return 0;
-            if (i >= shard_count) return m.numel;
-            const int64_t c = (int64_t)((__int128)m.numel * i / shard_count);
+            if (i >= count) return numel;
+            const int64_t c = (int64_t)((__int128)numel * i / count);
             return c / grain * grain;
         };
-        lo = cut(shard_index);
-        hi = cut(shard_index + 1);
+        lo = cut(index);
+        hi = cut(index + 1);
     }
     int chunk_of(int path) const { return chunk_paths > 0 ? path / chunk_paths : 0; }
 };
@@ -107,9 +116,13 @@ inline bool build_grid(Grid &g, int L, const int32_t *K, const int64_t *N, int P
         for (int l = 0; l < L; ++l)
             g.modules[g.module_id(l, g.table[(size_t)i * L + l])].members.push_back(i);
 
-    // partial-sum scratch for the modules whose paths span more than one chunk
+    // partial-sum scratch for the modules whose paths span more than one chunk; a slot for every
+    // module in the cast scratch (both kept 16-byte aligned for vector / bulk access)
     g.scratch_elems = 0;
+    g.cast_elems = 0;
     for (auto &m : g.modules) {
+        m.cast_off = g.cast_elems;
+        g.cast_elems += (m.numel + 7) / 8 * 8;
         m.partial_off = -1;
         if (g.num_chunks > 1 && !m.members.empty() &&
             g.chunk_of(m.members.front()) != g.chunk_of(m.members.back())) {
@@ -121,7 +134,7 @@ inline bool build_grid(Grid &g, int L, const int32_t *K, const int64_t *N, int P
     return true;
 }
 
-// Contributor set and coefficients of one module under a mask (step a0).
+// Contributor set and normalised coefficients of one module under a mask.
 struct ModuleCoeffs {
     std::vector<int> contributors; // ascending path ids in R(l,e)
     std::vector<float> coeff;      // w_i / W rounded to fp32 (normalised in double)
@@ -160,6 +173,7 @@ struct PassSpec {
     int64_t begin = 0, end = -1;   // element range of the module ([0, numel) when end < 0)
     float scale = 1.0f;            // factor on the finished outer gradient (used with PASS_UPDATE)
     bool second_moment = false;    // the update also reads and writes v (Adam family)
+    bool cast_out = false;         // cast(theta') is also stored in the module's cast-scratch slot
 };
 
 // Resident mode: one launch covers every module completely.
@@ -184,9 +198,13 @@ inline void plan_resident(const Grid &g, const std::vector<ModuleCoeffs> &mc,
     }
 }
 
-// Chunked mode, accumulate launch of chunk c.
+// Chunked mode, accumulate launch of chunk c.  The pass that sees a module's last reporting path
+// finishes the module and writes cast(theta') into the chunk's copies; with scatter_all (every
+// path copy is on the device: the one-call form) into every copy of the module, whatever its
+// chunk; with keep_cast also into the module's cast-scratch slot for later write-back launches.
 inline void plan_accumulate(const Grid &g, const std::vector<ModuleCoeffs> &mc, int c,
-                            std::vector<PassSpec> &out)
+                            std::vector<PassSpec> &out, bool scatter_all = false,
+                            bool keep_cast = false)
 {
     out.clear();
     for (size_t id = 0; id < g.modules.size(); ++id) {
@@ -210,8 +228,9 @@ inline void plan_accumulate(const Grid &g, const std::vector<ModuleCoeffs> &mc, 
         if (c == last) {
             p.flags |= PASS_UPDATE;
             p.second_moment = g.second_moment;
+            p.cast_out = keep_cast;
             for (int i : m.members)
-                if (g.chunk_of(i) == c) p.members.push_back(i);
+                if (scatter_all || g.chunk_of(i) == c) p.members.push_back(i);
         } else {
             p.flags |= PASS_PARTIAL_OUT;
         }
@@ -221,8 +240,10 @@ inline void plan_accumulate(const Grid &g, const std::vector<ModuleCoeffs> &mc, 
 
 // Chunked mode, write-back launch of chunk c: every slot of the chunk, or (skip_final) only
 // those that the accumulate launch of the same chunk did not already fill with the final value.
+// With use_cast the modules that were updated this round are filled from their cast-scratch slot
+// (path dtype) instead of from fp32 theta'.
 inline void plan_writeback(const Grid &g, const std::vector<ModuleCoeffs> &mc, int c, bool skip_final,
-                           std::vector<PassSpec> &out)
+                           std::vector<PassSpec> &out, bool use_cast = false)
 {
     out.clear();
     for (size_t id = 0; id < g.modules.size(); ++id) {
@@ -234,10 +255,28 @@ inline void plan_writeback(const Grid &g, const std::vector<ModuleCoeffs> &mc, i
         p.module = (int)id;
         g.shard_range(m, p.begin, p.end);
         if (p.begin >= p.end) continue;
-        p.flags = 0;
+        p.flags = (use_cast && k.update) ? PASS_CAST_IN : 0;
         for (int i : m.members)
             if (g.chunk_of(i) == c) p.members.push_back(i);
         if (p.members.empty()) continue;
+        out.push_back(std::move(p));
+    }
+}
+
+// One-call chunked mode: the modules that nobody updates this round (no reporting path, or zero
+// total weight) still hand cast(theta) to every one of their paths.
+inline void plan_refill_unchanged(const Grid &g, const std::vector<ModuleCoeffs> &mc,
+                                  std::vector<PassSpec> &out)
+{
+    for (size_t id = 0; id < g.modules.size(); ++id) {
+        const ModuleGeom &m = g.modules[id];
+        if (mc[id].update || m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
+        PassSpec p;
+        p.module = (int)id;
+        g.shard_range(m, p.begin, p.end);
+        if (p.begin >= p.end) continue;
+        p.flags = 0;
+        p.members = m.members;
         out.push_back(std::move(p));
     }
 }
@@ -252,8 +291,9 @@ struct Segment {
 // Bytes one element of a pass moves (cost model for balancing CTAs).
 inline double pass_cost_per_elem(const PassSpec &p, int elem_size)
 {
-    double c = 4.0; // theta read
+    double c = (p.flags & PASS_CAST_IN) ? (double)elem_size : 4.0; // cast slot, or theta, read
     c += (double)elem_size * (double)(p.contributors.size() + p.members.size());
+    if (p.cast_out) c += (double)elem_size;
     if (p.flags & PASS_UPDATE) c += 12.0;      // momentum read, theta' and m' written
     if ((p.flags & PASS_UPDATE) && p.second_moment) c += 8.0;  // v read and written
     if (p.flags & PASS_PARTIAL_IN) c += 4.0;

@@ -4,7 +4,6 @@
 #include "../../include/dipaco.h"
 
 #include <cmath>
-#include <mutex>
 
 #include "kernels.cuh"
 
@@ -13,9 +12,9 @@ using namespace dipaco;
 namespace {
 
 constexpr int STATIC_MAX_CHUNK = 32;   // path pointers carried in the kernel arguments
-constexpr int STATIC_MAX_DEVICES = 64;
 
-// Partial sums between chunks.  Every GPU that loads the library holds these 16 MiB until exit.
+// Partial sums between chunks.  Every GPU on which this module has been loaded (at the latest by
+// the first call of the entry point there) holds these 16 MiB until the process exits.
 static __device__ __align__(256) float g_static_partial[DIPACO_STATIC_MAX_NUMEL];
 
 struct StaticAccumulateArgs {
@@ -73,26 +72,27 @@ __global__ void __launch_bounds__(256) static_writeback_kernel(StaticWritebackAr
     }
 }
 
-std::mutex g_setup_mutex;
-float *g_partial_address[STATIC_MAX_DEVICES] = {};
-int g_sm_count[STATIC_MAX_DEVICES] = {};
-
-// Once per device, with that device current: the device address of the static array.  In host
-// code the array's name is only a handle for this look-up, never a pointer a kernel may use.
+// With that device current: the device address of the static array.  In host code the array's
+// name is only a handle for this look-up, never a pointer a kernel may use.  The look-up is
+// repeated on every call (it is cheap and allocates nothing once the module is loaded), so a
+// primary context that the application destroyed and re-created is followed.  The very first
+// look-up on a device makes the CUDA runtime load this file's module there, which is when the
+// array's 16 MiB are reserved: that can fail on a device whose memory is already exhausted.
 int static_setup(int device, float **partial, int *sm_count)
 {
-    std::lock_guard<std::mutex> lock(g_setup_mutex);
-    if (!g_partial_address[device]) {
-        void *addr = nullptr;
-        if (cudaGetSymbolAddress(&addr, g_static_partial) != cudaSuccess || !addr) return DIPACO_ECUDA;
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1)
-            return DIPACO_ECUDA;
-        g_partial_address[device] = static_cast<float *>(addr);
-        g_sm_count[device] = sms;
+    void *addr = nullptr;
+    const cudaError_t err = cudaGetSymbolAddress(&addr, g_static_partial);
+    if (err != cudaSuccess || !addr) {
+        cudaGetLastError();  // leave no sticky error behind for the caller's next runtime call
+        return err == cudaErrorMemoryAllocation ? DIPACO_ENOMEM : DIPACO_ECUDA;
     }
-    *partial = g_partial_address[device];
-    *sm_count = g_sm_count[device];
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) {
+        cudaGetLastError();
+        return DIPACO_ECUDA;
+    }
+    *partial = static_cast<float *>(addr);
+    *sm_count = sms;
     return DIPACO_OK;
 }
 
@@ -124,7 +124,7 @@ extern "C" int dipaco_module_sync_static(float *theta, float *momentum, int64_t 
     if (!theta || !momentum || !copy_ptrs || num_paths < 1 || numel < 0) return DIPACO_EINVAL;
     if (path_dtype != DIPACO_F32 && path_dtype != DIPACO_BF16) return DIPACO_EINVAL;
     if (chunk_paths < 1 || chunk_paths > STATIC_MAX_CHUNK) return DIPACO_EINVAL;
-    if (device < 0 || device >= STATIC_MAX_DEVICES) return DIPACO_EINVAL;
+    if (device < 0) return DIPACO_EINVAL;
     if (!std::isfinite(outer_lr) || !std::isfinite(outer_momentum)) return DIPACO_EINVAL;
     if (numel > (int64_t)DIPACO_STATIC_MAX_NUMEL) return DIPACO_ELIMIT;
     for (int i = 0; i < num_paths; ++i) {

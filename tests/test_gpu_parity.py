@@ -2,8 +2,9 @@
 
 Tolerance (fp32 results theta', m'): |gpu - oracle| <= 1e-6 * (1 + |oracle|).  Path copies must
 equal cast(gpu theta') bit for bit (fp32: the value itself; bf16: round-to-nearest-even) and, for
-bf16, lie within one bf16 rounding step plus the fp32 tolerance of the oracle's copy.  Kernel families, resident and chunked mode
-and repeated runs must agree bitwise.
+bf16, lie within one bf16 step (the exact spacing at the expected value) plus the fp32 tolerance
+of the oracle's copy (helpers.assert_bf16_copies_close).  Kernel families, resident and chunked
+mode and repeated runs must agree bitwise.
 """
 from __future__ import annotations
 
@@ -80,12 +81,7 @@ def assert_matches_oracle(pr, before, after, reported="cfg", weights="cfg", thre
 
 
 def assert_bf16_close(got_bits, want_bits):
-    """Two roundings of nearly equal fp32 values: at most one bf16 step (2^-7 relative) on top of
-    the fp32 tolerance (which dominates where theta' is close to zero)."""
-    got = helpers.bf16_bits_to_float(got_bits).astype(np.float64)
-    want = helpers.bf16_bits_to_float(want_bits).astype(np.float64)
-    bound = 1e-6 * (1.0 + np.abs(want)) + 2.0 ** -7 * np.abs(want)
-    assert np.all(np.abs(got - want) <= bound)
+    helpers.assert_bf16_copies_close(got_bits, want_bits)
 
 
 def assert_states_bitwise_equal(a, b):
@@ -167,13 +163,21 @@ def test_chunked_mode_is_bitwise_identical_to_resident(name):
         assert_states_bitwise_equal(resident, chunked)
 
 
-def test_incremental_api_with_fresh_buffers_for_writeback():
+@pytest.mark.parametrize("kernel", [B.DIPACO_KERNEL_AUTO, B.DIPACO_KERNEL_VECTOR, B.DIPACO_KERNEL_SCALAR])
+@pytest.mark.parametrize("empty_module", [False, True])
+def test_incremental_api_with_fresh_buffers_for_writeback(kernel, empty_module):
+    """The chunk API as a streaming caller uses it.  With bf16 copies the write-back launches read
+    cast(theta') from the scratch that the finishing passes filled; a module that nobody updated
+    has no entry there and is filled from theta."""
     base = synth.CONFIGS["grid16x16-masked"]
     pr = synth.make_problem(base.scaled(ALIGNED[3]), DEV)
+    if empty_module:
+        pr.reported = pr.reported.copy()
+        pr.reported[[i for i in range(256) if pr.table[i, 2] == 9]] = 0
     resident = clone_problem(pr)
     run_gpu(pr, resident)
     theta, momentum, paths = clone_problem(pr)
-    ctx = make_ctx(pr, chunk_paths=32)
+    ctx = make_ctx(pr, chunk_paths=32, kernel=kernel)
     nchunks, scratch = B.dipaco_plan_chunks(ctx)
     assert nchunks == 8 and scratch > 0
     B.dipaco_sync_begin(ctx, theta.data_ptr(), momentum.data_ptr(), pr.reported)
@@ -618,3 +622,155 @@ def test_adam_family_through_the_host_buffer_entry_point():
     for a, b in zip(host_paths, dev_paths):
         assert torch.equal(a.view(torch.int16), b.cpu().view(torch.int16))
     assert not torch.equal(host[2], second)
+
+
+def test_a_repeated_call_reuses_its_plan_and_any_change_replans():
+    """dipaco_outer_sync keeps the plan of the previous call while settings, buffers and mask stay
+    the same; whatever changes (mask, weights, a path buffer, theta) must give the result of a
+    fresh context."""
+    cfg = synth.CONFIGS["grid4x4"].scaled((3 * 4096 + 24, 4096 + 8, 2 * 4096 + 1003))
+    pr = synth.make_problem(cfg, DEV)
+
+    def fresh(reported, weights, order=None):
+        state = clone_problem(pr)
+        if order is not None:
+            state = (state[0], state[1], [state[2][i] for i in order])
+        run_gpu(pr, state, reported=reported, weights=weights)
+        return state
+
+    ctx = make_ctx(pr)
+    theta, momentum, paths = clone_problem(pr)
+
+    def restore():
+        theta.copy_(pr.theta); momentum.copy_(pr.momentum)
+        for p, q in zip(paths, pr.paths):
+            p.copy_(q)
+
+    def call(reported, bufs=None, th=None):
+        bufs = paths if bufs is None else bufs
+        th = theta if th is None else th
+        B.dipaco_outer_sync(ctx, th.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in bufs], reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+
+    for _ in range(3):                       # identical calls: the second and third reuse the plan
+        restore()
+        call(pr.reported)
+        assert_states_bitwise_equal((theta, momentum, paths), fresh(pr.reported, pr.weights))
+    mask = np.ones(16, dtype=np.uint8)
+    mask[[2, 11]] = 0
+    restore(); call(mask)                    # another mask
+    assert_states_bitwise_equal((theta, momentum, paths), fresh(mask, pr.weights))
+    restore(); call(None)                    # no mask
+    assert_states_bitwise_equal((theta, momentum, paths), fresh(None, pr.weights))
+    w2 = pr.weights[::-1].copy()
+    B.dipaco_set_weights(ctx, w2)            # other weights, same buffers and mask
+    restore(); call(None)
+    assert_states_bitwise_equal((theta, momentum, paths), fresh(None, w2))
+    restore()                                # same set of buffers bound to other paths
+    order = [1, 0] + list(range(2, 16))
+    swapped = [paths[i] for i in order]
+    for p, q in zip(swapped, pr.paths):
+        p.copy_(q)
+    call(None, bufs=swapped)
+    want = fresh(None, w2)
+    assert_states_bitwise_equal((theta, momentum, swapped), want)
+    other_theta = pr.theta.clone()           # another theta buffer
+    restore(); call(None, th=other_theta)
+    assert_states_bitwise_equal((other_theta, momentum, paths), fresh(None, w2))
+    B.dipaco_destroy(ctx)
+
+
+def test_a_wait_that_runs_out_is_reported_once_and_the_context_recovers():
+    """The time-out path end to end, without disturbing the pipeline kernels: the diagnostic
+    entry point makes one bounded wait (1 ms) run out on a barrier nothing completes.  The kernel
+    must end by itself, later launches must do nothing while the error is pending,
+    dipaco_device_status must report DIPACO_ETIMEOUT exactly once and re-arm the work counters,
+    and the next synchronisation must be bitwise correct."""
+    cfg = synth.CONFIGS["grid4x4"].scaled((6 * 4096 + 8, 4096 + 16, 2 * 4096 + 5))
+    pr = synth.make_problem(cfg, DEV)
+    ref = clone_problem(pr)
+    run_gpu(pr, ref)
+    for chunk in (0, 5):
+        ctx = make_ctx(pr, chunk_paths=chunk)
+        state = clone_problem(pr)
+        ptrs = [p.data_ptr() for p in state[2]]
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        B.dipaco_selftest_wait_expiry(ctx, 1_000_000)
+        end.record()
+        torch.cuda.synchronize()
+        ms = start.elapsed_time(end)
+        assert 0.9 <= ms < 100.0, "the wait should give up after about 1 ms, took %.3f ms" % ms
+        # the error is pending: this launch must leave everything as it is
+        B.dipaco_outer_sync(ctx, state[0].data_ptr(), state[1].data_ptr(), ptrs, pr.reported)
+        torch.cuda.synchronize()
+        assert_states_bitwise_equal(state, clone_problem(pr))
+        assert B.dipaco_device_status(ctx) == B.DIPACO_ETIMEOUT
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        # re-armed: the same call now does its work, and the work counters started from zero
+        B.dipaco_outer_sync(ctx, state[0].data_ptr(), state[1].data_ptr(), ptrs, pr.reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        assert_states_bitwise_equal(state, ref)
+        with pytest.raises(B.DipacoError):
+            B.dipaco_selftest_wait_expiry(ctx, 0)
+        B.dipaco_destroy(ctx)
+
+
+@pytest.mark.parametrize("mode", ["resident", "chunked", "host"])
+def test_compact_shards_match_the_oracle_and_the_unsharded_update(mode):
+    """Section 3.3, sharded executor: three executors that each hold ONLY their slab of theta,
+    momentum and of every path copy (separate allocations, packed) update it through their own
+    shard context; the slabs put back side by side equal the oracle's result for the whole
+    problem and, bit for bit, the unsharded call."""
+    cfg = synth.SyncConfig("shards", (1, 4, 4), (5 * 8192 + 4096 + 24, 3 * 8192 + 8, 2 * 8192 + 1003),
+                           "bf16", weights="tokens", momentum_std=1e-4, mask_prob=0.2, seed=11)
+    pr = synth.make_problem(cfg, DEV)
+    before = host_state(clone_problem(pr))
+    unsharded = clone_problem(pr)
+    run_gpu(pr, unsharded)
+    whole = make_ctx(pr, chunk_paths=0 if mode == "resident" else 5)
+    B.dipaco_device_status(whole)
+    S, L = 3, cfg.num_levels
+    lvl, mod = pr.level_offsets(), pr.module_offsets()
+    out = clone_problem(pr)
+    where = "cpu" if mode == "host" else DEV
+
+    def module_slices(bounds):
+        for l, k in enumerate(cfg.modules_per_level):
+            for e in range(k):
+                base = int(mod[l]) + e * cfg.level_numel[l]
+                yield slice(base + bounds[l][0], base + bounds[l][1])
+
+    def path_slices(bounds):
+        for l in range(L):
+            yield slice(int(lvl[l]) + bounds[l][0], int(lvl[l]) + bounds[l][1])
+
+    for s_idx in range(S):
+        bounds = [B.dipaco_plan_shard(whole, s_idx, S, l) for l in range(L)]
+        theta_s = torch.cat([pr.theta[sl] for sl in module_slices(bounds)]).to(where)
+        mom_s = torch.cat([pr.momentum[sl] for sl in module_slices(bounds)]).to(where)
+        paths_s = [torch.cat([p[sl] for sl in path_slices(bounds)]).to(where) for p in pr.paths]
+        if mode == "host":
+            theta_s, mom_s = theta_s.pin_memory(), mom_s.pin_memory()
+            paths_s = [p.pin_memory() for p in paths_s]
+        ctx = B.dipaco_create_shard(whole, s_idx, S, 0)
+        fn = B.dipaco_outer_sync_host if mode == "host" else B.dipaco_outer_sync
+        fn(ctx, theta_s.data_ptr(), mom_s.data_ptr(), [p.data_ptr() for p in paths_s], pr.reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        B.dipaco_destroy(ctx)
+        pos = 0
+        for sl in module_slices(bounds):
+            n = sl.stop - sl.start
+            out[0][sl] = theta_s[pos:pos + n].to(DEV)
+            out[1][sl] = mom_s[pos:pos + n].to(DEV)
+            pos += n
+        for i, p in enumerate(paths_s):
+            pos = 0
+            for sl in path_slices(bounds):
+                n = sl.stop - sl.start
+                out[2][i][sl] = p[pos:pos + n].to(DEV)
+                pos += n
+    B.dipaco_destroy(whole)
+    assert_states_bitwise_equal(out, unsharded)
+    assert_matches_oracle(pr, before, out)

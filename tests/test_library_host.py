@@ -1,4 +1,5 @@
-"""CPU tests of the CUDA library's host side: exported symbols, validation, planning (step a0).
+"""CPU tests of the CUDA library's host side: exported symbols, validation, and planning (the
+contributor sets and coefficients).
 
 No compute call is made: contexts are created plan-only (device = -1)."""
 from __future__ import annotations
@@ -224,11 +225,25 @@ def test_planned_traffic_of_resident_mode_is_the_algorithmic_minimum():
         nbytes, launches = B.dipaco_plan_traffic(ctx, r)
         assert launches == 1 and nbytes == synth.algorithmic_bytes(cfg, r)
         B.dipaco_destroy(ctx)
-    # walking the 16x16 workload in chunks of 32 paths carries partial sums: ~1.5x the traffic
+    # Walking the 16x16 workload in chunks of 32 paths: one launch per chunk.  On top of the
+    # algorithmic bytes every launch but the last reads theta again and carries the fp32 partial
+    # sum of the modules whose paths span chunks (the shared block and the 16 last-level modules:
+    # 850e6 parameters): theta re-read 7 times, partial written 7 times and read 7 times.
     cfg = synth.CONFIGS["grid16x16"]
     ctx = plan_ctx(cfg, chunk_paths=32)
     nbytes, launches = B.dipaco_plan_traffic(ctx)
-    assert launches == 15 and 1.4 < nbytes / synth.algorithmic_bytes(cfg) < 1.6
+    spanning = 17 * 50_000_000
+    assert launches == 8
+    assert nbytes == synth.algorithmic_bytes(cfg) + spanning * 4 * (7 + 7 + 7)
+    assert nbytes < 252e9
+    B.dipaco_destroy(ctx)
+    # a module that nobody updates is refilled inside the first launch: no extra launch
+    cfg = synth.CONFIGS["grid16x16-masked"]
+    ctx = plan_ctx(cfg, chunk_paths=32, weights=synth.path_weights(cfg))
+    r = synth.reported_mask(cfg).copy()
+    r[[i for i in range(256) if synth.path_table(cfg.modules_per_level)[i, 1] == 3]] = 0
+    nbytes, launches = B.dipaco_plan_traffic(ctx, r)
+    assert launches == 8
     B.dipaco_destroy(ctx)
 
 
@@ -246,6 +261,46 @@ def test_shards_partition_the_planned_traffic():
         with pytest.raises(B.DipacoError):
             B.dipaco_set_shard(ctx, *bad)
     B.dipaco_destroy(ctx)
+
+
+def test_compact_shard_contexts_tile_the_problem_exactly_once():
+    """dipaco_plan_shard / dipaco_create_shard (Section 3.3, sharded executor): over the shards
+    every element of every level is owned exactly once, a shard context is the same grid with the
+    slab sizes as module sizes, and the planned traffic of the shards sums to the whole's."""
+    cfg = synth.CONFIGS["grid16x16-masked"].scaled((100_003, 8192 * 5, 8191))
+    w = synth.path_weights(cfg)
+    r = synth.reported_mask(cfg)
+    whole = plan_ctx(cfg, weights=w)
+    total, _ = B.dipaco_plan_traffic(whole, r)
+    S = 3
+    parts = 0
+    for l, n in enumerate(cfg.level_numel):
+        cuts = [B.dipaco_plan_shard(whole, s, S, l) for s in range(S)]
+        assert cuts[0][0] == 0 and cuts[-1][1] == n
+        for (a0, b0), (a1, b1) in zip(cuts, cuts[1:]):
+            assert b0 == a1 and a0 <= b0 and a1 <= b1
+        assert all(a % 8192 == 0 for a, _ in cuts)
+    for s in range(S):
+        ctx = B.dipaco_create_shard(whole, s, S, device=-1)
+        for l in range(cfg.num_levels):
+            a, b = B.dipaco_plan_shard(whole, s, S, l)
+            for e in (0, cfg.modules_per_level[l] - 1):
+                _, _, numel = B.dipaco_plan_offsets(ctx, l, e)
+                assert numel == b - a
+        # same contributor sets and coefficients as the whole problem
+        for (l, e) in ((0, 0), (1, 5), (2, 15)):
+            got = B.dipaco_plan_module(ctx, l, e, cfg.num_paths, r)
+            want = B.dipaco_plan_module(whole, l, e, cfg.num_paths, r)
+            for x, y in zip(got[:3], want[:3]):
+                np.testing.assert_array_equal(x, y)
+        parts += B.dipaco_plan_traffic(ctx, r)[0]
+        B.dipaco_destroy(ctx)
+    assert parts == total
+    with pytest.raises(B.DipacoError):
+        B.dipaco_create_shard(whole, 3, 3, device=-1)
+    with pytest.raises(B.DipacoError):
+        B.dipaco_plan_shard(whole, 0, 3, 7)
+    B.dipaco_destroy(whole)
 
 
 def test_a_c99_program_can_use_the_library(tmp_path):

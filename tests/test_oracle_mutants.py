@@ -38,6 +38,7 @@ MUTANTS = [
     ("module offset inside theta not advanced", "            module_base += n;\n        }\n        level_base",
      "            module_base += 0;\n        }\n        level_base"),
     ("bf16 cast truncates", "if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u)))", "if (0)"),
+    ("bf16 cast rounds a NaN like a number", "if ((bits & 0x7fffffffu) > 0x7f800000u)", "if (0)"),
     ("bf16 ties round away from zero", "(lower == 0x8000u && (upper & 1u))", "(lower == 0x8000u)"),
     ("learning rate applied twice to momentum", "t1 = t0 - outer_lr * (delta + outer_momentum * m1);",
      "t1 = t0 - outer_lr * (delta + outer_lr * outer_momentum * m1);"),

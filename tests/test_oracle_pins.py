@@ -420,6 +420,28 @@ def test_bf16_cast_is_round_to_nearest_even_like_the_library_cast():
     np.testing.assert_array_equal(ps[0], helpers.float_to_bf16_bits_torch(vals))
 
 
+def test_bf16_cast_of_nan_is_a_nan_whatever_its_payload():
+    """A NaN module value reaches the copies as a NaN: never as an infinity (what rounding the
+    bit pattern like a number gives when the payload sits in the low 16 bits only) and never as a
+    finite value.  Which NaN (sign, payload) is not specified, exactly as for the library cast,
+    which returns its canonical quiet NaN."""
+    bits = np.array([0x7fc00000, 0xffc00000, 0x7f800001, 0xff800001, 0x7f80ffff, 0x7fffffff,
+                     0x7f808000, 0x7fa00000, 0xffffffff, 0x7fc00001], dtype=np.uint32)
+    vals = bits.view(np.float32)
+    assert np.all(np.isnan(vals))
+    n = vals.size
+    cfg = synth.SyncConfig("nan", (1,), (n,), "bf16")
+    table = np.zeros((1, 1), dtype=np.int32)
+    # nobody reports: theta is kept and every copy receives cast(theta)
+    th, mo, ps = helpers.run_oracle(cfg, table, vals, np.zeros(n, np.float32),
+                                    [np.zeros(n, np.uint16)], None, np.zeros(1, np.uint8))
+    np.testing.assert_array_equal(th.view(np.uint32), bits)
+    out = ps[0].astype(np.uint32)
+    assert np.all((out & 0x7f80) == 0x7f80) and np.all((out & 0x007f) != 0)
+    lib = helpers.bf16_bits_to_float(helpers.float_to_bf16_bits_torch(vals))
+    assert np.all(np.isnan(lib)) and np.all(np.isnan(helpers.bf16_bits_to_float(ps[0])))
+
+
 def test_threads_do_not_change_the_result():
     cfg = tiny_cfg((1, 2, 2), (1000, 777, 513), "bf16", momentum_std=1e-3, seed=18)
     pr = synth.make_problem(cfg)
