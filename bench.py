@@ -653,6 +653,7 @@ def run_e2e(args, cfg, problem, make_ctx, world, device):
                               pin_memory=True)
     except RuntimeError as exc:
         return {"value": None, "unit": UNIT, "error": "could not pin host memory: %s" % exc}
+    pcie = pcie_probe(paths_h, device)
     dst = 0
     for l, k in enumerate(cfg.modules_per_level):
         for e in range(k):
@@ -703,8 +704,50 @@ def run_e2e(args, cfg, problem, make_ctx, world, device):
            "d2h_bytes_per_step": 8 * small.module_params + small.num_paths * small.params_per_path * es,
            "api": "dipaco_outer_sync_host, pinned host buffers, slab-ordered streaming, staging "
                   "bounded by %d path copies" % chunk}
+    if pcie:
+        # what this box's PCIe link gives a plain pinned copy, measured in this process: the
+        # step cannot be faster than the bytes of the busier direction at the both-ways rate
+        busier = max(out["h2d_bytes_per_step"], out["d2h_bytes_per_step"])
+        ideal_ms = busier / (pcie["both_ways_each_gbs"] * 1e9) * 1e3
+        pcie["ideal_ms_per_step"] = ideal_ms
+        pcie["frac_of_ideal"] = ideal_ms / ms_max
+        out["pcie"] = pcie
     if note:
         out["reduced"] = note
+    return out
+
+
+def pcie_probe(pinned, device, nbytes=2 << 30, reps=3):
+    """GB/s of plain pinned copies on this machine: host->device alone, device->host alone and both at
+    once (per direction), on 2 GiB pieces of the (not yet filled) pinned block of the end-to-end leg."""
+    import torch
+    flat = pinned.view(-1).view(torch.uint8)
+    if flat.numel() < 2 * nbytes:
+        return None
+    try:
+        dev_in = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        dev_out = torch.zeros(nbytes, dtype=torch.uint8, device=device)
+    except RuntimeError:
+        return None
+    up, down = torch.cuda.Stream(device), torch.cuda.Stream(device)
+
+    def run(do_up, do_down):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            if do_up:
+                with torch.cuda.stream(up):
+                    dev_in.copy_(flat[:nbytes], non_blocking=True)
+            if do_down:
+                with torch.cuda.stream(down):
+                    flat[nbytes:2 * nbytes].copy_(dev_out, non_blocking=True)
+        torch.cuda.synchronize()
+        return nbytes * reps / (time.perf_counter() - t0) / 1e9
+
+    run(True, True)
+    out = {"h2d_gbs": run(True, False), "d2h_gbs": run(False, True), "both_ways_each_gbs": run(True, True)}
+    del dev_in, dev_out
+    torch.cuda.empty_cache()
     return out
 
 

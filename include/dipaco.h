@@ -146,8 +146,10 @@ int dipaco_sync_end(dipaco_ctx *ctx);
  * cast in one fused pass, and the result is copied back into theta, momentum and the slot of
  * every path of the module while the next slab is already being uploaded.  Device staging is
  * bounded by the size of chunk_paths path copies (> 0 required) plus theta and momentum.  Paths
- * that did not report are not uploaded.  Results are bitwise those of dipaco_outer_sync.
- * Synchronous: returns when all host buffers hold the result.
+ * that did not report are not uploaded.  Path copies that lie equally spaced in host memory
+ * (rows of one allocation) are moved with one strided copy per slab instead of one per path.
+ * Results are bitwise those of dipaco_outer_sync.  Synchronous: returns when all host buffers
+ * hold the result, and on an error only after every copy it started has finished.
  */
 int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
                            void *const *path_ptrs_host, const uint8_t *reported,
@@ -263,15 +265,18 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
  * Tuning of the bulk-copy kernel's dynamic scheduling: a launch is cut into work items (runs of
  * tiles of one module) that the persistent CTAs draw from a counter.  An item moves at most
  * max_item_bytes of traffic (default 2 MiB) and a launch is cut into at least items_per_cta
- * items per CTA (default 16) so that the CTAs finish together.  0 keeps a value.  Results do not
+ * items per CTA (default 64) so that the CTAs finish together.  0 keeps a value.  Results do not
  * depend on the cut.
  */
 int dipaco_set_work_items(dipaco_ctx *ctx, int64_t max_item_bytes, int32_t items_per_cta);
 
 /*
- * Tuning of dipaco_outer_sync_host: the most bytes of path data one streamed unit uploads
- * (0 = no cap other than the staging buffers).  Smaller units fill and drain the pipeline
- * faster, larger ones mean fewer and larger copies.
+ * Tuning of dipaco_outer_sync_host: the most bytes of path data that one streamed unit stages
+ * on the device in each direction (0 = the default, 512 MiB; always at least one tile of every
+ * copy of the module, at most 1/6 of chunk_paths path copies).  The download of a unit cannot
+ * start before the unit is uploaded and reduced, so a call takes about one unit's transfer time
+ * longer than the PCIe transfer itself: smaller units shorten that, larger ones mean fewer and
+ * larger copies.
  */
 int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes);
 

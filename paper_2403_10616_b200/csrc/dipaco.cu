@@ -62,9 +62,9 @@ struct dipaco_ctx {
     int ctas_per_sm = 1, stages = 10, units = 2;  // bulk-copy kernel tuning (measured on B200)
     int io_slots = 3;                            // buffers of theta/momentum/result tiles
     int64_t item_bytes = 2 * 1024 * 1024;        // most traffic of one dynamic work item
-    int items_per_cta = 16;                      // least number of items per CTA that a launch is cut into
+    int items_per_cta = 64;                      // least number of items per CTA that a launch is cut into
     int64_t launches = 0;
-    int64_t host_unit_bytes = (int64_t)1 << 40;  // upload size cap of one unit in host mode
+    int64_t host_unit_bytes = (int64_t)512 << 20;  // staged bytes (each way) of one unit in host mode
 
     void *dev_tables = nullptr;
     size_t dev_tables_capacity = 0;
@@ -762,7 +762,7 @@ int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes)
     if (!ctx || bytes < 0) return DIPACO_EINVAL;
     if (ctx->state != STATE_IDLE) return DIPACO_ESTATE;
     ++ctx->settings_version;
-    ctx->host_unit_bytes = bytes == 0 ? (int64_t)1 << 40 : bytes;
+    ctx->host_unit_bytes = bytes == 0 ? (int64_t)512 << 20 : bytes;
     return DIPACO_OK;
 }
 
