@@ -256,7 +256,9 @@ int dipaco_set_kernel(dipaco_ctx *ctx, int32_t kernel);
  * the shared memory of the chosen layout is rejected with DIPACO_EINVAL and nothing changes;
  * result buffers beyond two are dropped at launch while they would leave the ring shallower than a
  * launch of that mix of modules needs (10 stages when most elements have 8 or more contributors,
- * 6 otherwise).
+ * 6 otherwise).  A launch that stages more fp32 tiles per buffer than the layout was accepted
+ * for (the second moment of an Adam-family optimiser selected later) falls back to the next
+ * smaller tile that fits; results do not depend on any of this.
  */
 int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages,
                       int32_t units_per_thread, int32_t io_slots);

@@ -35,6 +35,7 @@ struct PackedLaunch {
     size_t bulk_segs_off = 0, bulk_first_off = 0, rag_segs_off = 0, rag_first_off = 0;
     int bulk_ctas = 0, rag_ctas = 0;
     int io_arrays = 2;
+    int units = 2;                        // 16-byte units per compute thread and tile of this launch
     bool aligned_kernel_is_vector = false;
     int num_passes = 0, total_items = 0;  // dynamic scheduling of the bulk-copy kernel
     double mean_contributors = 0.0;       // per element of the bulk range
@@ -139,31 +140,50 @@ int tile_units(const dipaco_ctx *ctx)
     return ctx->units > 0 ? ctx->units : 2;
 }
 
-int64_t tile_elems(const dipaco_ctx *ctx)
+// Elements of one tile of `units` 16-byte units per compute thread.
+int64_t tile_elems_of(const dipaco_ctx *ctx, int units)
 {
     const int ue = ctx->dtype == DIPACO_BF16 ? 8 : 4;
-    return (int64_t)BULK_COMPUTE_THREADS * ue * tile_units(ctx);
+    return (int64_t)BULK_COMPUTE_THREADS * ue * units;
 }
 
-// Shared memory of one bulk-kernel CTA for a given depth.
-size_t bulk_smem_bytes(const dipaco_ctx *ctx, int stages, int io_arrays, int io_slots)
+// The tile of the configured tuning (launches that need more fp32 tiles per buffer than fit may
+// fall back to a smaller one, which always divides this one).
+int64_t tile_elems(const dipaco_ctx *ctx)
 {
-    const size_t tile = (size_t)tile_elems(ctx);
+    return tile_elems_of(ctx, tile_units(ctx));
+}
+
+// Shared memory of one bulk-kernel CTA for a given tile and depth.
+size_t bulk_smem_bytes(const dipaco_ctx *ctx, int units, int stages, int io_arrays, int io_slots)
+{
+    const size_t tile = (size_t)tile_elems_of(ctx, units);
     const size_t stage = tile * ctx->elem_size;
     size_t bytes = (size_t)stages * stage + (size_t)io_slots * io_arrays * tile * 4;
     if (ctx->elem_size != 4) bytes += (size_t)io_slots * stage;
     return bytes + sizeof(BulkShared) + 128;
 }
 
-int pick_stages(const dipaco_ctx *ctx, int io_arrays, int io_slots)
+int pick_stages(const dipaco_ctx *ctx, int units, int io_arrays, int io_slots)
 {
     const size_t budget =
         std::min(SMEM_LIMIT, SMEM_PER_SM / (size_t)ctx->ctas_per_sm - 2 * SMEM_CTA_RESERVE);
     int best = 0;
     for (int s = 2; s <= BULK_MAX_STAGES; ++s)
-        if (bulk_smem_bytes(ctx, s, io_arrays, io_slots) <= budget) best = s;
+        if (bulk_smem_bytes(ctx, units, s, io_arrays, io_slots) <= budget) best = s;
     if (ctx->stages > 0) return ctx->stages <= best ? ctx->stages : best;
     return best;
+}
+
+// Units per thread for a launch that stages io_arrays fp32 tiles per buffer: the configured
+// value, or the next smaller one that still leaves a ring of two stages beside two buffers
+// (the partial sum of a chunk walk and the second moment of the Adam family each add a tile
+// that the tuning may not have been chosen for).  0 = nothing fits.
+int fit_units(const dipaco_ctx *ctx, int io_arrays)
+{
+    for (int nu = tile_units(ctx); nu >= 1; nu /= 2)
+        if (pick_stages(ctx, nu, io_arrays, 2) >= 2) return nu;
+    return 0;
 }
 
 struct PtrLookup {
@@ -192,8 +212,13 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     std::vector<void *> members;
     std::vector<int64_t> bulk_begin(specs.size(), 0), bulk_end(specs.size(), 0);
     std::vector<int64_t> rag_begin(specs.size(), 0), rag_end(specs.size(), 0);
-    const int64_t tile = tile_elems(ctx);
     bool any_partial = false;
+    for (const PassSpec &sp : specs)
+        if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
+    const int io_arrays = (any_partial ? 3 : 2) + (ctx->optimizer == DIPACO_OPT_ADAM ? 1 : 0);
+    const int units = ctx->kernel == DIPACO_KERNEL_AUTO ? fit_units(ctx, io_arrays) : tile_units(ctx);
+    if (units < 1) return DIPACO_EINVAL;
+    const int64_t tile = tile_elems_of(ctx, units);
 
     for (size_t i = 0; i < specs.size(); ++i) {
         const PassSpec &sp = specs[i];
@@ -211,7 +236,6 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         pd.bulk_end = 0;
         if ((sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) && (m.partial_off < 0 || !ctx->partial))
             return DIPACO_ESTATE;
-        if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
         if (((sp.flags & PASS_CAST_IN) || sp.cast_out) && !ctx->cast_scratch) return DIPACO_ESTATE;
         bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
                        ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
@@ -320,7 +344,8 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     out.rag_first_off = append(rag_first.data(), rag_first.size() * sizeof(int32_t));
     out.bulk_ctas = bulk_ctas;
     out.rag_ctas = rag_ctas;
-    out.io_arrays = (any_partial ? 3 : 2) + (ctx->optimizer == DIPACO_OPT_ADAM ? 1 : 0);
+    out.io_arrays = io_arrays;
+    out.units = units;
     out.aligned_kernel_is_vector = vector_kernel;
     out.num_passes = (int)passes.size();
     out.total_items = (int)total_items;
@@ -392,7 +417,7 @@ int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages,
     return cudaGetLastError() == cudaSuccess ? DIPACO_OK : DIPACO_ECUDA;
 }
 
-int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays,
+int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays, int nu,
                 double mean_contributors, cudaStream_t stream)
 {
     // Shared memory is split between the ring of path tiles and the theta/momentum/result
@@ -401,11 +426,10 @@ int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays
     const int wanted = ctx->stages > 0 ? std::min(ctx->stages, 10) : 10;
     const int min_stages = mean_contributors >= 8.0 ? wanted : std::min(wanted, 6);
     int io_slots = ctx->io_slots;
-    while (io_slots > 2 && pick_stages(ctx, io_arrays, io_slots) < min_stages) --io_slots;
-    const int stages = pick_stages(ctx, io_arrays, io_slots);
+    while (io_slots > 2 && pick_stages(ctx, nu, io_arrays, io_slots) < min_stages) --io_slots;
+    const int stages = pick_stages(ctx, nu, io_arrays, io_slots);
     if (stages < 2) return DIPACO_EINVAL;
-    const size_t smem = bulk_smem_bytes(ctx, stages, io_arrays, io_slots);
-    const int nu = tile_units(ctx);
+    const size_t smem = bulk_smem_bytes(ctx, nu, stages, io_arrays, io_slots);
     const int col = nu == 1 ? 0 : (nu == 2 ? 1 : 2);
     if (ctx->dtype == DIPACO_BF16) {
         if (nu == 1) return launch_bulk_t<__nv_bfloat16, 1>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
@@ -460,7 +484,7 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
                 sync_direct_kernel<float, 8><<<pl.bulk_ctas, 256, 0, stream>>>(lp);
             if (cudaGetLastError() != cudaSuccess) rc = DIPACO_ECUDA;
         } else {
-            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, pl.mean_contributors, stream);
+            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, pl.units, pl.mean_contributors, stream);
         }
         if (rc != DIPACO_OK) return rc;
         ++ctx->launches;
@@ -735,7 +759,8 @@ int dipaco_set_tuning(dipaco_ctx *ctx, int32_t ctas_per_sm, int32_t stages, int3
     ctx->stages = 0;
     // chunked contexts stage a third fp32 tile (the partial sum) per buffer
     const int io_arrays = (ctx->grid.num_chunks > 1 ? 3 : 2) + (ctx->optimizer == DIPACO_OPT_ADAM ? 1 : 0);
-    const bool fits = pick_stages(ctx, io_arrays, 2) >= 2 && (!stages || stages <= pick_stages(ctx, io_arrays, 2));
+    const int nu = tile_units(ctx);
+    const bool fits = pick_stages(ctx, nu, io_arrays, 2) >= 2 && (!stages || stages <= pick_stages(ctx, nu, io_arrays, 2));
     if (!fits) {
         ctx->ctas_per_sm = old_ctas;
         ctx->units = old_units;

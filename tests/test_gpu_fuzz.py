@@ -1,6 +1,8 @@
 """Seeded random structures against the oracle: grids, path subsets, sizes around tile and 16-byte
 boundaries, weights with zeros, masks that empty whole modules, chunk sizes, kernel families,
-tunings, rescaling, local levels and optimisers, all through the C ABI."""
+tunings, rescaling, local levels and optimisers, and the way the synchronisation is carried out
+(one call, the same call repeated on restored inputs, the chunk API with fresh write-back buffers,
+host buffers, compact shards), all through the C ABI."""
 from __future__ import annotations
 
 import numpy as np
@@ -16,7 +18,7 @@ pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
 SIZES = [0, 1, 3, 7, 8, 9, 64, 1000, 2047, 2048, 2056, 4095, 4096, 4100, 4104, 8192, 8200, 12288 + 24,
-         20000, 4096 * 5 + 8, 4096 * 3 + 1003]
+         20000, 4096 * 5 + 8, 4096 * 3 + 1003, 3 * 8192 + 1003, 2 * 8192, 5 * 8192 + 24]
 
 
 def random_case(seed):
@@ -56,10 +58,73 @@ def random_case(seed):
         "input_kind": int(rng.rand() < 0.25),
         "misalign": bool(rng.rand() < 0.2),
     }
+    # drawn last, so the structures of the earlier seeds stay what they were
+    opts["route"] = str(rng.choice(["one_call", "one_call", "repeat", "chunk_api", "host", "shards"]))
+    opts["shards"] = int(rng.randint(2, 4))
+    if opts["route"] in ("chunk_api", "host") and opts["chunk"] == 0:
+        opts["chunk"] = int(rng.choice([1, 2, 5, 32]))
+    if opts["route"] == "shards":
+        opts["misalign"] = False
     return K, numel, table, dtype, weights, reported, opts
 
 
-@pytest.mark.parametrize("seed", range(64))
+def configure(ctx, opts, second):
+    """Apply the drawn options to a context; returns the oracle's Adam tuple (or None)."""
+    B.dipaco_set_kernel(ctx, opts["kernel"])
+    try:
+        B.dipaco_set_tuning(ctx, *opts["tuning"])
+    except B.DipacoError as exc:                   # a layout that does not fit shared memory
+        assert exc.status == B.DIPACO_EINVAL
+    B.dipaco_set_module_scale(ctx, opts["scale"])
+    B.dipaco_set_level_sync(ctx, opts["level_sync"])
+    adam = None
+    if opts["optimizer"] == 3:
+        b1, b2, eps, wd, step = opts["adam"]
+        B.dipaco_set_adam(ctx, second.data_ptr(), b1, b2, eps, wd, step)
+        f = lambda x: float(np.float32(x))
+        adam = (f(b1), f(b2), f(eps), f(wd), 1 - f(b1) ** step if step else 1.0,
+                1 - f(b2) ** step if step else 1.0)
+    else:
+        B.dipaco_set_optimizer(ctx, opts["optimizer"])
+    B.dipaco_set_input_kind(ctx, opts["input_kind"])
+    return adam
+
+
+def run_route(ctx, opts, cfg, table, reported, theta, momentum, second, paths):
+    """Carry the synchronisation out the drawn way, in place on the given tensors."""
+    route = opts["route"]
+    ptrs = [p.data_ptr() for p in paths]
+    if route == "one_call":
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), ptrs, reported)
+    elif route == "repeat":
+        saved = (theta.clone(), momentum.clone(), second.clone(), [p.clone() for p in paths])
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), ptrs, reported)
+        torch.cuda.synchronize()
+        theta.copy_(saved[0]); momentum.copy_(saved[1]); second.copy_(saved[2])
+        for p, q in zip(paths, saved[3]):
+            p.copy_(q)
+        B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), ptrs, reported)   # plan reused
+    elif route == "chunk_api":
+        chunk = opts["chunk"]
+        nchunks, _ = B.dipaco_plan_chunks(ctx)
+        B.dipaco_sync_begin(ctx, theta.data_ptr(), momentum.data_ptr(), reported)
+        for c in range(nchunks):
+            stage = [p.clone() for p in paths[c * chunk:(c + 1) * chunk]]
+            B.dipaco_sync_accumulate(ctx, c, [p.data_ptr() for p in stage])
+            torch.cuda.synchronize()
+            del stage
+        for c in range(nchunks):
+            mine = paths[c * chunk:(c + 1) * chunk]
+            if opts["level_sync"] is None:         # (levels kept local keep their contents)
+                for p in mine:
+                    p.fill_(float("nan"))          # write-back must not depend on the old contents
+            B.dipaco_sync_writeback(ctx, c, [p.data_ptr() for p in mine])
+        B.dipaco_sync_end(ctx)
+    else:
+        raise AssertionError(route)
+
+
+@pytest.mark.parametrize("seed", range(96))
 def test_random_structure_matches_the_oracle(seed):
     K, numel, table, dtype, weights, reported, opts = random_case(seed)
     cfg = synth.SyncConfig("fuzz%d" % seed, tuple(K), tuple(numel), dtype, momentum_std=1e-4, seed=seed)
@@ -69,6 +134,7 @@ def test_random_structure_matches_the_oracle(seed):
     momentum = torch.empty(cfg.module_params, device=DEV).normal_(0, 1e-4, generator=gen)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     mod_off = np.concatenate([[0], np.cumsum([k * n for k, n in zip(K, numel)])])
+    lvl_off = np.concatenate([[0], np.cumsum(numel)])
     paths, keepalive = [], []
     for i in range(table.shape[0]):
         parts = [theta[int(mod_off[l]) + int(table[i, l]) * n:int(mod_off[l]) + (int(table[i, l]) + 1) * n]
@@ -81,35 +147,66 @@ def test_random_structure_matches_the_oracle(seed):
             keepalive.append(back)
             row = view
         paths.append(row)
-    pr = synth.SyncProblem(cfg, np.ascontiguousarray(table, dtype=np.int32), weights, reported, theta,
-                           momentum, paths)
-    before = host_state((theta, momentum, paths))
-
-    code = B.DIPACO_BF16 if dtype == "bf16" else B.DIPACO_F32
-    ctx = B.dipaco_create(K, numel, pr.table, weights, np.float32(0.7), np.float32(0.9), code,
-                          opts["chunk"], 0)
-    B.dipaco_set_kernel(ctx, opts["kernel"])
-    try:
-        B.dipaco_set_tuning(ctx, *opts["tuning"])
-    except B.DipacoError as exc:                   # a layout that does not fit shared memory
-        assert exc.status == B.DIPACO_EINVAL
-    B.dipaco_set_module_scale(ctx, opts["scale"])
-    B.dipaco_set_level_sync(ctx, opts["level_sync"])
+    table = np.ascontiguousarray(table, dtype=np.int32)
     second = torch.empty_like(theta).normal_(0, 1e-4, generator=gen).abs_()
     v_host = helpers.tensor_to_numpy(second)
-    adam = None
-    if opts["optimizer"] == 3:
-        b1, b2, eps, wd, step = opts["adam"]
-        B.dipaco_set_adam(ctx, second.data_ptr(), b1, b2, eps, wd, step)
-        f = lambda x: float(np.float32(x))
-        adam = (f(b1), f(b2), f(eps), f(wd), 1 - f(b1) ** step if step else 1.0,
-                1 - f(b2) ** step if step else 1.0)
+    before = host_state((theta, momentum, paths))
+    code = B.DIPACO_BF16 if dtype == "bf16" else B.DIPACO_F32
+    ctx = B.dipaco_create(K, numel, table, weights, np.float32(0.7), np.float32(0.9), code, opts["chunk"], 0)
+    route = opts["route"]
+
+    if route == "host":
+        # everything lives in host memory (the path copies in one pinned block or one by one)
+        theta, momentum, second = theta.cpu().pin_memory(), momentum.cpu().pin_memory(), second.cpu().pin_memory()
+        if seed % 2:
+            block = torch.stack([p.cpu() for p in paths]).pin_memory()
+            paths = [block[i] for i in range(len(paths))]
+        else:
+            paths = [p.cpu() for p in paths]
+        adam = configure(ctx, opts, second)
+        B.dipaco_outer_sync_host(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths],
+                                 reported)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    elif route == "shards":
+        # S executors, each with its own packed slabs (Section 3.3); results put back side by side
+        adam = configure(ctx, opts, second)
+        S = opts["shards"]
+        for s_idx in range(S):
+            bounds = [B.dipaco_plan_shard(ctx, s_idx, S, l) for l in range(len(K))]
+            mods = [slice(int(mod_off[l]) + e * numel[l] + bounds[l][0], int(mod_off[l]) + e * numel[l] + bounds[l][1])
+                    for l in range(len(K)) for e in range(K[l])]
+            lvls = [slice(int(lvl_off[l]) + bounds[l][0], int(lvl_off[l]) + bounds[l][1]) for l in range(len(K))]
+            th_s = torch.cat([theta[sl] for sl in mods])
+            mo_s = torch.cat([momentum[sl] for sl in mods])
+            v_s = torch.cat([second[sl] for sl in mods])
+            ps_s = [torch.cat([p[sl] for sl in lvls]) for p in paths]
+            if th_s.numel() == 0:
+                continue
+            shard = B.dipaco_create_shard(ctx, s_idx, S, 0)
+            if opts["optimizer"] == 3:
+                B.dipaco_set_adam(shard, v_s.data_ptr(), *opts["adam"])
+            B.dipaco_outer_sync(shard, th_s.data_ptr(), mo_s.data_ptr(), [p.data_ptr() for p in ps_s], reported)
+            assert B.dipaco_device_status(shard) == B.DIPACO_OK
+            B.dipaco_destroy(shard)
+            pos = 0
+            for sl in mods:
+                n = sl.stop - sl.start
+                theta[sl] = th_s[pos:pos + n]; momentum[sl] = mo_s[pos:pos + n]; second[sl] = v_s[pos:pos + n]
+                pos += n
+            for p, q in zip(paths, ps_s):
+                pos = 0
+                for sl in lvls:
+                    n = sl.stop - sl.start
+                    p[sl] = q[pos:pos + n]
+                    pos += n
     else:
-        B.dipaco_set_optimizer(ctx, opts["optimizer"])
-    B.dipaco_set_input_kind(ctx, opts["input_kind"])
-    B.dipaco_outer_sync(ctx, theta.data_ptr(), momentum.data_ptr(), [p.data_ptr() for p in paths], reported)
-    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        adam = configure(ctx, opts, second)
+        run_route(ctx, opts, cfg, table, reported, theta, momentum, second, paths)
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
     B.dipaco_destroy(ctx)
+    pr = synth.SyncProblem(cfg, table, weights, reported, theta, momentum, paths)
+
+
 
     scale64 = None if opts["scale"] is None else opts["scale"].astype(np.float64)
     want_th, want_mo, want_ps = helpers.run_oracle(cfg, pr.table, *before, weights, reported,
