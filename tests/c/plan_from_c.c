@@ -54,6 +54,31 @@ int main(void)
         printf("outer_sync should have refused\n");
         return 1;
     }
+    /* two executors that each hold half of every module (Section 3.3): slab bounds and the
+     * plan-only context of executor 1 of a grid large enough to be cut at the 8192 grain */
+    {
+        const int64_t big_numel[3] = {40000, 16384, 100};
+        dipaco_ctx *whole = NULL, *half = NULL;
+        int64_t a = -1, b = -1, n = -1;
+        if (dipaco_create(&whole, 3, modules_per_level, big_numel, 4, table, weights, 0.7f, 0.9f,
+                          DIPACO_BF16, 0, -1) != DIPACO_OK)
+            return 1;
+        if (dipaco_plan_shard(whole, 0, 2, 0, &a, &b) != DIPACO_OK || a != 0 || b != 16384 ||
+            dipaco_plan_shard(whole, 1, 2, 0, &a, &b) != DIPACO_OK || a != 16384 || b != 40000 ||
+            dipaco_plan_shard(whole, 1, 2, 2, &a, &b) != DIPACO_OK || a != 0 || b != 100 ||
+            dipaco_plan_shard(whole, 2, 2, 0, &a, &b) != DIPACO_EINVAL) {
+            printf("plan_shard mismatch\n");
+            return 1;
+        }
+        if (dipaco_create_shard(&half, whole, 1, 2, -1) != DIPACO_OK || !half ||
+            dipaco_plan_offsets(half, 0, 0, NULL, NULL, &n) != DIPACO_OK || n != 40000 - 16384 ||
+            dipaco_plan_offsets(half, 1, 1, &theta_off, &path_off, &n) != DIPACO_OK || n != 8192 ||
+            theta_off != (40000 - 16384) + 8192 || path_off != 40000 - 16384) {
+            printf("create_shard mismatch\n");
+            return 1;
+        }
+        if (dipaco_destroy(whole) != DIPACO_OK || dipaco_destroy(half) != DIPACO_OK) return 1;
+    }
     if (strcmp(dipaco_strerror(DIPACO_ENODEV), "unknown status") == 0) return 1;
     if (dipaco_destroy(ctx) != DIPACO_OK) return 1;
     printf("ok\n");
