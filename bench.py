@@ -39,7 +39,7 @@ REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the referen
 # digest is checked and "traffic" is null after any change to them.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9918
 NCU_CAPTURE_SOURCES = ("kernels.cuh", "dipaco.cu", "plan.hpp")
-NCU_CAPTURE_SOURCES_SHA256 = "d7052c6774385bf8dace2ef3e465b9c4d11c21b3beee727db0e0d97d12a1ff7a"
+NCU_CAPTURE_SOURCES_SHA256 = "5d6c0146077d8e204bfa4593d70e9841a12820d60366dba880852f9dcec57db3"
 NCU_CAPTURE_COMMAND = ("ncu --set full --clock-control none -k regex:sync_bulk_kernel -s 3 -c 3 "
                        "python bench.py --level-numel 2000000 --steps 3 --warmup 3 --no-e2e "
                        "--no-chunked --no-cpu-baseline --no-variants --no-other-workloads")
