@@ -76,6 +76,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--host-unit-mb", type=int, default=0,
                     help="cap on the upload of one streamed unit of the host-buffer leg (0 = default)")
+    ap.add_argument("--host-threads", type=int, default=-1,
+                    help="host threads that fan each module's result out to its paths in the "
+                         "host-buffer leg (-1 = library default, 0 = none: one download per path)")
     ap.add_argument("--items-per-cta", type=int, default=0)
     ap.add_argument("--item-kb", type=int, default=0)
     ap.add_argument("--no-other-workloads", action="store_true")
@@ -682,6 +685,7 @@ def run_e2e(args, cfg, problem, make_ctx, world, device):
 
     if args.host_unit_mb:
         B.dipaco_set_host_unit_bytes(ctx, args.host_unit_mb << 20)
+    B.dipaco_set_host_threads(ctx, args.host_threads)
     step()   # warm-up: allocates the staging buffers
     steps = max(1, args.e2e_steps)
     barrier(world)
@@ -698,17 +702,31 @@ def run_e2e(args, cfg, problem, make_ctx, world, device):
     ms_max, units = aggregate(dt_ms, float(small.path_params), world, device)
     n_rep = small.num_paths if problem.reported is None else int(problem.reported.sum())
     B.dipaco_destroy(ctx)
+    results_bytes = 8 * small.module_params + small.num_paths * small.params_per_path * es
+    if args.host_threads != 0:
+        # the new value of a module crosses PCIe once; host threads copy it into every path
+        d2h = (8 + es) * small.module_params
+    else:
+        d2h = results_bytes
     out = {"value": units / (ms_max * 1e-3), "unit": UNIT, "ms_per_step": ms_max, "steps": steps,
            "ms_per_step_min": min(per_step), "ms_per_step_mean": sum(per_step) / len(per_step),
            "h2d_bytes_per_step": 8 * small.module_params + n_rep * small.params_per_path * es,
-           "d2h_bytes_per_step": 8 * small.module_params + small.num_paths * small.params_per_path * es,
+           "d2h_bytes_per_step": d2h,
+           "host_result_bytes_per_step": results_bytes,
            "api": "dipaco_outer_sync_host, pinned host buffers, slab-ordered streaming, staging "
-                  "bounded by %d path copies" % chunk}
+                  "bounded by %d path copies; %s" % (
+                      chunk, "every path copy downloaded" if args.host_threads == 0 else
+                      "each module's new value downloaded once and copied into its paths by host threads")}
     if pcie:
         # what this box's PCIe link gives a plain pinned copy, measured in this process: the
         # step cannot be faster than the bytes of the busier direction at the both-ways rate
-        busier = max(out["h2d_bytes_per_step"], out["d2h_bytes_per_step"])
-        ideal_ms = busier / (pcie["both_ways_each_gbs"] * 1e9) * 1e3
+        # (both directions equally loaded: the both-ways rate; otherwise each at its one-way rate)
+        if out["d2h_bytes_per_step"] >= 0.8 * out["h2d_bytes_per_step"]:
+            busier = max(out["h2d_bytes_per_step"], out["d2h_bytes_per_step"])
+            ideal_ms = busier / (pcie["both_ways_each_gbs"] * 1e9) * 1e3
+        else:
+            ideal_ms = max(out["h2d_bytes_per_step"] / pcie["h2d_gbs"],
+                           out["d2h_bytes_per_step"] / pcie["d2h_gbs"]) / 1e9 * 1e3
         pcie["ideal_ms_per_step"] = ideal_ms
         pcie["frac_of_ideal"] = ideal_ms / ms_max
         out["pcie"] = pcie

@@ -148,7 +148,8 @@ int dipaco_sync_end(dipaco_ctx *ctx);
  * bounded by the size of chunk_paths path copies (> 0 required) plus theta and momentum.  Paths
  * that did not report are not uploaded.  Path copies that lie equally spaced in host memory
  * (rows of one allocation) are moved with one strided copy per slab instead of one per path.
- * Results are bitwise those of dipaco_outer_sync.  Synchronous: returns when all host buffers
+ * By default a pool of host threads fans each module's result out to its paths
+ * (dipaco_set_host_threads).  Results are bitwise those of dipaco_outer_sync.  Synchronous: returns when all host buffers
  * hold the result, and on an error only after every copy it started has finished.
  */
 int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
@@ -281,6 +282,19 @@ int dipaco_set_work_items(dipaco_ctx *ctx, int64_t max_item_bytes, int32_t items
  * larger copies.
  */
 int dipaco_set_host_unit_bytes(dipaco_ctx *ctx, int64_t bytes);
+
+/*
+ * Host threads of dipaco_outer_sync_host.  Every path of a module receives the same
+ * cast(theta'), so with threads > 0 each streamed piece of it is downloaded once, into a pinned
+ * buffer of the library, and `threads` host threads copy it into the slot of every path while
+ * later pieces are still being uploaded: PCIe carries one copy per module instead of one per
+ * path.  The threads belong to the context (created by the first call that needs them, joined
+ * by dipaco_destroy) and sleep between calls.  0 = no host threads: the device writes one copy
+ * per path and all of them are downloaded.  -1 = the default (half the hardware threads, at
+ * most 4: more of them compete with the uploads for host memory bandwidth).  Results are
+ * identical either way.
+ */
+int dipaco_set_host_threads(dipaco_ctx *ctx, int32_t threads);
 
 /*
  * Synchronise the context's last stream and report what the kernels recorded: DIPACO_OK, or

@@ -50,7 +50,7 @@ EXPORTS = [
     "dipaco_set_host_unit_bytes", "dipaco_plan_traffic", "dipaco_set_module_scale",
     "dipaco_set_level_sync", "dipaco_set_shard", "dipaco_set_optimizer", "dipaco_set_adam",
     "dipaco_set_input_kind", "dipaco_plan_shard", "dipaco_create_shard",
-    "dipaco_selftest_wait_expiry", "dipaco_set_work_items",
+    "dipaco_selftest_wait_expiry", "dipaco_set_work_items", "dipaco_set_host_threads",
 ]
 
 _lib = None
@@ -96,6 +96,7 @@ def load() -> ctypes.CDLL:
     lib.dipaco_set_kernel.argtypes = [vp, i32]
     lib.dipaco_set_tuning.argtypes = [vp, i32, i32, i32, i32]
     lib.dipaco_set_work_items.argtypes = [vp, i64, i32]
+    lib.dipaco_set_host_threads.argtypes = [vp, i32]
     lib.dipaco_device_status.argtypes = [vp]
     lib.dipaco_set_host_unit_bytes.argtypes = [vp, i64]
     lib.dipaco_launch_count.argtypes = [vp]
@@ -280,6 +281,10 @@ def dipaco_set_tuning(ctx, ctas_per_sm=0, stages=0, units_per_thread=0, io_slots
 def dipaco_set_work_items(ctx, max_item_bytes=0, items_per_cta=0) -> None:
     _check(load().dipaco_set_work_items(ctx, int(max_item_bytes), int(items_per_cta)),
            "dipaco_set_work_items")
+
+
+def dipaco_set_host_threads(ctx, threads: int) -> None:
+    _check(load().dipaco_set_host_threads(ctx, int(threads)), "dipaco_set_host_threads")
 
 
 def dipaco_set_host_unit_bytes(ctx, nbytes: int) -> None:

@@ -16,7 +16,7 @@ DEPENDS = ["dipaco.cu", "static_sync.cu", "kernels.cuh", "plan.hpp", "host_mode.
 def nvcc_command(out, verbose=False):
     cmd = ["nvcc", "-std=c++17", "-O3", "-lineinfo",
            "-gencode", "arch=compute_100a,code=sm_100a",
-           "-Xcompiler", "-fPIC,-O2,-Wall", "-shared", "-cudart", "static",
+           "-Xcompiler", "-fPIC,-O2,-Wall,-pthread", "-shared", "-cudart", "static",
            "-o", out]
     if verbose:
         cmd += ["-Xptxas", "-v"]

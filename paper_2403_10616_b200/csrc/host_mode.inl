@@ -9,12 +9,17 @@
 //     kernel  the resident-mode pass on [a, b), reading the staged rows, writing theta', m' in
 //             place and cast(theta') once per path of the module into the rows of an output buffer
 //     D2H     theta'[a:b], m'[a:b], and each output row into its path's slot
-// Three streams (upload, kernel, download) and a ring of three buffer pairs overlap the upload of
-// later units with the kernel and the download of earlier ones.  Both PCIe directions carry the
-// same number of bytes and the download of a unit can only start once the unit is uploaded and
-// reduced, so a step takes (bytes one way / PCIe rate) + about one unit's transfer time: units
-// are kept small (dipaco_set_host_unit_bytes, 512 MiB each way by default), whatever the
-// module's size.  Everything a unit's kernel needs besides the data (its tables) is uploaded
+// Streams for upload, kernel and download and a ring of three buffer sets overlap the upload of
+// later units with the kernel and the download of earlier ones.  The download of a unit can only
+// start once the unit is uploaded and reduced, so a step takes (bytes of the busier direction /
+// PCIe rate) + about one unit's transfer time: units are kept small (dipaco_set_host_unit_bytes,
+// 512 MiB by default), whatever the module's size.
+// Every path of a module receives the SAME cast(theta').  With host threads (dipaco_set_host_threads,
+// on by default) that piece crosses PCIe once per unit, into a small pinned bounce buffer, and a
+// pool of host threads copies it into the slot of every path while later units upload: the
+// device->host traffic shrinks from one copy per path to one per module, and the upload, which
+// cannot shrink (every reporting copy is different data), has the link almost to itself.  With
+// zero host threads the kernel writes one output row per path and all of them are downloaded.  Everything a unit's kernel needs besides the data (its tables) is uploaded
 // once, before the first unit, so no small copy queues behind the bulk uploads.  Pieces of path
 // copies that lie equally spaced in host memory (copies carved from one allocation) move as one
 // strided 2-D copy per run instead of one copy per path.  Staging memory: at most chunk_paths
@@ -24,6 +29,113 @@
 namespace {
 
 constexpr int HOST_BUFFERS = 3;
+constexpr size_t HOST_BOUNCE_BYTES = (size_t)64 << 20;  // pinned landing buffer of one unit's cast piece
+
+// Copy for destinations that will not be read again soon: streaming (non-temporal) stores write
+// whole cache lines without first reading them, which halves the memory traffic of the fan-out
+// and leaves more of the host's memory bandwidth to the PCIe uploads running beside it.
+inline void copy_streaming(char *dst, const char *src, size_t n)
+{
+#if defined(__SSE2__)
+    if (reinterpret_cast<uintptr_t>(dst) % 16 == 0) {
+        size_t i = 0;
+        for (; i + 64 <= n; i += 64) {
+            const __m128i a = _mm_loadu_si128(reinterpret_cast<const __m128i *>(src + i));
+            const __m128i b = _mm_loadu_si128(reinterpret_cast<const __m128i *>(src + i + 16));
+            const __m128i c = _mm_loadu_si128(reinterpret_cast<const __m128i *>(src + i + 32));
+            const __m128i d = _mm_loadu_si128(reinterpret_cast<const __m128i *>(src + i + 48));
+            _mm_stream_si128(reinterpret_cast<__m128i *>(dst + i), a);
+            _mm_stream_si128(reinterpret_cast<__m128i *>(dst + i + 16), b);
+            _mm_stream_si128(reinterpret_cast<__m128i *>(dst + i + 32), c);
+            _mm_stream_si128(reinterpret_cast<__m128i *>(dst + i + 48), d);
+        }
+        if (i < n) std::memcpy(dst + i, src + i, n - i);
+        _mm_sfence();  // streaming stores are weakly ordered: make them visible before completion is signalled
+        return;
+    }
+#endif
+    std::memcpy(dst, src, n);
+}
+
+// A pool of host threads that copies one source piece into many destinations.  run() is called
+// from a CUDA host-function callback (no CUDA call is made in here): thread t copies byte range t
+// of T of the piece into every destination, so its share of the source stays in its cache.
+class ReplicatePool {
+public:
+    struct Job {
+        const char *src = nullptr;
+        size_t bytes = 0;
+        std::vector<char *> dst;
+    };
+    explicit ReplicatePool(int threads)
+    {
+        for (int t = 0; t < threads; ++t) workers_.emplace_back([this, t, threads] { work(t, threads); });
+    }
+    ~ReplicatePool()
+    {
+        {
+            std::lock_guard<std::mutex> lock(mutex_);
+            stop_ = true;
+        }
+        wake_.notify_all();
+        for (std::thread &w : workers_) w.join();
+    }
+    int size() const { return (int)workers_.size(); }
+    void run(const Job &job)
+    {
+        std::unique_lock<std::mutex> lock(mutex_);
+        job_ = &job;
+        remaining_ = (int)workers_.size();
+        ++generation_;
+        wake_.notify_all();
+        done_.wait(lock, [this] { return remaining_ == 0; });
+        job_ = nullptr;
+    }
+
+private:
+    void work(int t, int threads)
+    {
+        unsigned long long seen = 0;
+        for (;;) {
+            const Job *job;
+            {
+                std::unique_lock<std::mutex> lock(mutex_);
+                wake_.wait(lock, [&] { return stop_ || generation_ != seen; });
+                if (stop_) return;
+                seen = generation_;
+                job = job_;
+            }
+            // shares cut at 64-byte boundaries
+            const size_t lines = (job->bytes + 63) / 64;
+            const size_t lo = std::min(job->bytes, lines * (size_t)t / threads * 64);
+            const size_t hi = std::min(job->bytes, lines * (size_t)(t + 1) / threads * 64);
+            if (hi > lo)
+                for (char *d : job->dst) copy_streaming(d + lo, job->src + lo, hi - lo);
+            {
+                std::lock_guard<std::mutex> lock(mutex_);
+                if (--remaining_ == 0) done_.notify_all();
+            }
+        }
+    }
+    std::vector<std::thread> workers_;
+    std::mutex mutex_;
+    std::condition_variable wake_, done_;
+    const Job *job_ = nullptr;
+    unsigned long long generation_ = 0;
+    int remaining_ = 0;
+    bool stop_ = false;
+};
+
+struct ReplicateCall {
+    ReplicatePool *pool;
+    ReplicatePool::Job job;
+};
+
+void CUDART_CB replicate_callback(void *data)
+{
+    ReplicateCall *call = static_cast<ReplicateCall *>(data);
+    call->pool->run(call->job);
+}
 
 // One streamed unit: elements [a, b) of one module.
 struct HostUnit {
@@ -38,7 +150,11 @@ struct HostMode {
     char *stage_out[HOST_BUFFERS] = {};               // rows: cast(theta') for every path of the module
     size_t stage_bytes = 0;                           // size of each of those buffers
     size_t max_pitch = 0;                             // largest pitch a 2-D copy accepts
+    char *bounce[HOST_BUFFERS] = {};                  // pinned host: one unit's cast piece lands here
+    ReplicatePool *pool = nullptr;                    // host threads that fan the piece out
     cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    cudaStream_t fan_stream = nullptr;                // carries the host-function callbacks
+    cudaEvent_t fan_done[HOST_BUFFERS] = {};          // piece copied to every path: bounce reusable
     cudaEvent_t in_ready[HOST_BUFFERS] = {};     // upload of the unit in this buffer finished
     cudaEvent_t kernel_done[HOST_BUFFERS] = {};  // kernel finished: input reusable, output ready
     cudaEvent_t out_done[HOST_BUFFERS] = {};     // download finished: output buffer reusable
@@ -61,6 +177,14 @@ void host_mode_release(dipaco_ctx *ctx)
     if (!h) return;
     if (h->in_stream) cudaStreamSynchronize(h->in_stream);
     if (h->out_stream) cudaStreamSynchronize(h->out_stream);
+    if (h->fan_stream) cudaStreamSynchronize(h->fan_stream);
+    delete h->pool;
+    h->pool = nullptr;
+    for (int b = 0; b < HOST_BUFFERS; ++b) {
+        if (h->bounce[b]) cudaFreeHost(h->bounce[b]);
+        if (h->fan_done[b]) cudaEventDestroy(h->fan_done[b]);
+    }
+    if (h->fan_stream) cudaStreamDestroy(h->fan_stream);
     if (h->theta_d) cudaFree(h->theta_d);
     if (h->momentum_d) cudaFree(h->momentum_d);
     if (h->second_d) cudaFree(h->second_d);
@@ -95,9 +219,11 @@ int host_mode_prepare(dipaco_ctx *ctx)
     bool ok = cudaDeviceGetAttribute(&pitch, cudaDevAttrMaxPitch, ctx->device) == cudaSuccess &&
               cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&h->out_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&h->fan_stream, cudaStreamNonBlocking) == cudaSuccess &&
               cudaEventCreateWithFlags(&h->main_ready, cudaEventDisableTiming) == cudaSuccess;
     for (int b = 0; ok && b < HOST_BUFFERS; ++b)
-        ok = cudaEventCreateWithFlags(&h->in_ready[b], cudaEventDisableTiming) == cudaSuccess &&
+        ok = cudaEventCreateWithFlags(&h->fan_done[b], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&h->in_ready[b], cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&h->kernel_done[b], cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&h->out_done[b], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
@@ -109,15 +235,19 @@ int host_mode_prepare(dipaco_ctx *ctx)
     return DIPACO_OK;
 }
 
-// Rows of a unit: one per reporting copy on the way in, one per path of the module on the way out.
-size_t host_unit_rows(const dipaco_ctx *ctx, size_t id)
+// Staged rows of a unit: one per reporting copy on the way in; on the way out one per path of the
+// module, or a single one when host threads fan it out.
+size_t host_unit_rows(const dipaco_ctx *ctx, size_t id, bool fan_out)
 {
-    return std::max<size_t>(std::max(ctx->coeffs[id].contributors.size(), ctx->grid.modules[id].members.size()), 1);
+    const size_t in = ctx->coeffs[id].contributors.size();
+    const size_t out = fan_out ? 1 : ctx->grid.modules[id].members.size();
+    return std::max<size_t>(std::max(in, out), 1);
 }
 
 // Cut the round into units of at most `cap` staged bytes each way (but at least one tile of every
-// row), starting on tile boundaries.  Returns the bytes one staging buffer has to hold.
-size_t plan_host_units(const dipaco_ctx *ctx, size_t cap, std::vector<HostUnit> &units)
+// row), starting on tile boundaries; with fan-out a unit's piece also has to fit the bounce
+// buffer.  Returns the bytes one staging buffer has to hold.
+size_t plan_host_units(const dipaco_ctx *ctx, size_t cap, bool fan_out, std::vector<HostUnit> &units)
 {
     const Grid &g = ctx->grid;
     const int es = ctx->elem_size;
@@ -127,9 +257,11 @@ size_t plan_host_units(const dipaco_ctx *ctx, size_t cap, std::vector<HostUnit> 
     for (size_t id = 0; id < g.modules.size(); ++id) {
         const ModuleGeom &m = g.modules[id];
         if (m.members.empty() || m.numel == 0 || !g.synced(m)) continue;
-        const size_t rows = host_unit_rows(ctx, id);
+        const size_t rows = host_unit_rows(ctx, id, fan_out);
         // a tile's bytes are a multiple of the 256-byte row stride
-        const int64_t slab = std::max<int64_t>(tile, (int64_t)(cap / (rows * (size_t)es)) / tile * tile);
+        size_t fit = cap / (rows * (size_t)es);
+        if (fan_out) fit = std::min(fit, HOST_BOUNCE_BYTES / (size_t)es);
+        const int64_t slab = std::max<int64_t>(tile, (int64_t)fit / tile * tile);
         int64_t lo = 0, hi = m.numel;
         g.shard_range(m, lo, hi);
         for (int64_t a = lo; a < hi; a += slab) {
@@ -234,9 +366,24 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
     // at most chunk_paths path copies
     const size_t bound = (size_t)g.chunk_paths * (size_t)g.params_per_path * es / (2 * HOST_BUFFERS);
     const size_t cap = std::max<size_t>(std::min(bound, (size_t)ctx->host_unit_bytes), 256);
+    const bool fan_out = ctx->host_threads > 0;
     std::vector<HostUnit> units;
-    const size_t need = plan_host_units(ctx, cap, units);
+    const size_t need = plan_host_units(ctx, cap, fan_out, units);
     if (units.empty()) return DIPACO_OK;
+    if (fan_out) {
+        if (h->pool && h->pool->size() != ctx->host_threads) {
+            if (cudaStreamSynchronize(h->fan_stream) != cudaSuccess) return DIPACO_ECUDA;
+            delete h->pool;
+            h->pool = nullptr;
+        }
+        if (!h->pool) h->pool = new ReplicatePool(ctx->host_threads);
+        for (int b = 0; b < HOST_BUFFERS; ++b)
+            if (!h->bounce[b] && cudaMallocHost(&h->bounce[b], HOST_BOUNCE_BYTES) != cudaSuccess) {
+                cudaGetLastError();
+                h->bounce[b] = nullptr;
+                return DIPACO_ENOMEM;
+            }
+    }
     if (need > h->stage_bytes) {
         if (cudaStreamSynchronize(h->in_stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess ||
             cudaStreamSynchronize(h->out_stream) != cudaSuccess)
@@ -255,6 +402,7 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
     // Whatever way this function is left from here on, no copy may still be running into (or out
     // of) the caller's host buffers: the call is synchronous, and after an error the caller is
     // free to release them at once.
+    std::vector<ReplicateCall> fan_calls(units.size());  // outlive the callbacks: declared before the drain
     struct DrainOnExit {
         HostMode *h;
         cudaStream_t main;
@@ -263,6 +411,7 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
             cudaStreamSynchronize(h->in_stream);
             cudaStreamSynchronize(main);
             cudaStreamSynchronize(h->out_stream);
+            cudaStreamSynchronize(h->fan_stream);
         }
     } drain{h, stream};
 
@@ -293,7 +442,7 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
         sp.begin = a;
         sp.end = b;
         reqs[u].specs.push_back(std::move(sp));
-        std::vector<void *> rows(m.members.size());
+        std::vector<void *> rows(fan_out ? 1 : m.members.size());
         for (size_t j = 0; j < rows.size(); ++j)
             rows[j] = reinterpret_cast<void *>(reinterpret_cast<uintptr_t>(h->stage_out[buf] + j * pitch) -
                                                (uintptr_t)a * es);
@@ -313,7 +462,8 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
     // the side streams must not run ahead of work queued earlier on the caller's stream
     if (cudaEventRecord(h->main_ready, stream) != cudaSuccess ||
         cudaStreamWaitEvent(h->in_stream, h->main_ready, 0) != cudaSuccess ||
-        cudaStreamWaitEvent(h->out_stream, h->main_ready, 0) != cudaSuccess)
+        cudaStreamWaitEvent(h->out_stream, h->main_ready, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(h->fan_stream, h->main_ready, 0) != cudaSuccess)
         return DIPACO_ECUDA;
 
     std::vector<char *> host_rows;
@@ -375,13 +525,34 @@ int host_mode_sync(dipaco_ctx *ctx, float *theta_host, float *momentum_host,
         }
         host_rows.clear();
         for (int i : m.members) host_rows.push_back(static_cast<char *>(path_ptrs_host[i]) + slot_off);
-        rc = copy_rows(false, h->stage_out[buf], pitch, host_rows, piece, h->max_pitch, h->out_stream);
-        if (rc != DIPACO_OK) return rc;
-        if (cudaEventRecord(h->out_done[buf], h->out_stream) != cudaSuccess) return DIPACO_ECUDA;
+        if (!fan_out || host_rows.size() == 1) {
+            // one output row per path (or the only path's row) straight into place
+            rc = copy_rows(false, h->stage_out[buf], pitch, host_rows, piece, h->max_pitch, h->out_stream);
+            if (rc != DIPACO_OK) return rc;
+            if (cudaEventRecord(h->out_done[buf], h->out_stream) != cudaSuccess) return DIPACO_ECUDA;
+        } else {
+            // the single output row lands in the bounce buffer (once the fan-out that last used it
+            // is done) and host threads copy it into every path's slot
+            if (u >= HOST_BUFFERS && cudaStreamWaitEvent(h->out_stream, h->fan_done[buf], 0) != cudaSuccess)
+                return DIPACO_ECUDA;
+            if (cudaMemcpyAsync(h->bounce[buf], h->stage_out[buf], piece, cudaMemcpyDeviceToHost,
+                                h->out_stream) != cudaSuccess ||
+                cudaEventRecord(h->out_done[buf], h->out_stream) != cudaSuccess ||
+                cudaStreamWaitEvent(h->fan_stream, h->out_done[buf], 0) != cudaSuccess)
+                return DIPACO_ECUDA;
+            ReplicateCall &call = fan_calls[u];
+            call.pool = h->pool;
+            call.job.src = h->bounce[buf];
+            call.job.bytes = piece;
+            call.job.dst = host_rows;
+            if (cudaLaunchHostFunc(h->fan_stream, replicate_callback, &call) != cudaSuccess) return DIPACO_ECUDA;
+        }
+        if (fan_out && cudaEventRecord(h->fan_done[buf], h->fan_stream) != cudaSuccess) return DIPACO_ECUDA;
     }
     if (cudaStreamSynchronize(h->in_stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess ||
-        cudaStreamSynchronize(h->out_stream) != cudaSuccess)
+        cudaStreamSynchronize(h->out_stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->fan_stream) != cudaSuccess)
         return DIPACO_ECUDA;
     return DIPACO_OK;
 }

@@ -331,8 +331,11 @@ def test_host_buffers_entry_point_matches_the_oracle(name, pinned):
         paths = [p.pin_memory() for p in paths]
     chunk = 32 if cfg.num_paths > 32 else 5
     ctx = make_ctx(pr, chunk_paths=chunk)
-    for rnd in range(2):            # second call reuses the staging buffers
-        if rnd == 1:
+    # default: host threads fan each module's result out to its paths; then the same with three
+    # threads and with none (one output row per path, all downloaded); later calls reuse the staging
+    for rnd, threads in enumerate((-1, 3, 0)):
+        B.dipaco_set_host_threads(ctx, threads)
+        if rnd > 0:
             theta.copy_(pr.theta); momentum.copy_(pr.momentum)
             for p, q in zip(paths, pr.paths):
                 p.copy_(q)
