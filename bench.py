@@ -473,6 +473,32 @@ def run_ours(args):
                              "value": cfg.path_params / (ms_c * 1e-3), "unit": UNIT,
                              "effective_gbs": alg_bytes / (ms_c * 1e-3) / 1e9,
                              "gpu_launches": int(B.dipaco_launch_count(ctx) - before)}
+        # the same walk through the chunk API, as a caller that holds one chunk at a time drives
+        # it: accumulate every chunk in order, then a write-back launch per chunk
+        nchunks, _ = B.dipaco_plan_chunks(ctx)
+        cp = cfg.chunk_paths
+        chunk_arrs = [B.ptr_array(ptrs[c * cp:(c + 1) * cp]) for c in range(nchunks)]
+
+        def api_step():
+            B.dipaco_sync_begin(ctx, theta_ptr, momentum_ptr, problem.reported, stream_handle)
+            for c in range(nchunks):
+                B.dipaco_sync_accumulate(ctx, c, chunk_arrs[c])
+            for c in range(nchunks):
+                B.dipaco_sync_writeback(ctx, c, chunk_arrs[c])
+            B.dipaco_sync_end(ctx)
+
+        try:
+            api_step()
+            before = B.dipaco_launch_count(ctx)
+            api_steps = max(3, min(args.steps, 8))
+            ms_api, _ = time_steps(api_step, api_steps, 1)
+            result["chunked"]["chunk_api"] = {
+                "ms_per_step": ms_api, "steps": api_steps,
+                "gpu_launches": int(B.dipaco_launch_count(ctx) - before),
+                "note": "dipaco_sync_begin / accumulate x%d / writeback x%d / end over the same "
+                        "buffers; write-back launches read the bf16 cast scratch" % (nchunks, nchunks)}
+        except B.DipacoError as exc:
+            result["chunked"]["chunk_api"] = {"error": str(exc)}
         B.dipaco_destroy(ctx)
 
     # ---- CPU oracle on a slab of the same inputs (rank 0, N = 1)

@@ -777,3 +777,36 @@ def test_compact_shards_match_the_oracle_and_the_unsharded_update(mode):
     B.dipaco_destroy(whole)
     assert_states_bitwise_equal(out, unsharded)
     assert_matches_oracle(pr, before, out)
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other():
+    """Contexts share nothing (tables, counters, error word and scratch are per context): two
+    synchronisations queued back to back on different streams, so that they overlap on the
+    device, each give bitwise their own result."""
+    cfgs = [synth.CONFIGS["grid4x4"].scaled((24 * 4096 + 8, 8 * 4096 + 16, 8 * 4096)),
+            synth.CONFIGS["grid16x16-masked"].scaled((4 * 4096 + 72, 2 * 4096 + 8, 4096 + 1003))]
+    problems = [synth.make_problem(c, DEV) for c in cfgs]
+    refs = []
+    for pr, chunk in zip(problems, (0, 32)):
+        ref = clone_problem(pr)
+        run_gpu(pr, ref, chunk_paths=chunk)
+        refs.append(ref)
+    states = [clone_problem(pr) for pr in problems]
+    ctxs = [make_ctx(problems[0], 0), make_ctx(problems[1], 32)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for pr, st, ctx, stream in zip(problems, states, ctxs, streams):
+            B.dipaco_outer_sync(ctx, st[0].data_ptr(), st[1].data_ptr(), [p.data_ptr() for p in st[2]],
+                                pr.reported, stream=stream)
+        for stream in streams:
+            stream.synchronize()
+        for pr, st, ref in zip(problems, states, refs):
+            assert_states_bitwise_equal(st, ref)
+            st[0].copy_(pr.theta); st[1].copy_(pr.momentum)      # restore for the next repetition
+            for p, q in zip(st[2], pr.paths):
+                p.copy_(q)
+        torch.cuda.synchronize()
+    for ctx in ctxs:
+        assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+        B.dipaco_destroy(ctx)

@@ -263,6 +263,30 @@ def test_shards_partition_the_planned_traffic():
     B.dipaco_destroy(ctx)
 
 
+def test_tuning_setters_validate_their_arguments():
+    ctx = plan_ctx(synth.CONFIGS["grid2x2"], chunk_paths=2)
+    for good in ((0, 0), (1 << 20, 32), (0, 4096)):
+        B.dipaco_set_work_items(ctx, *good)
+    for bad in ((-1, 0), (0, -1), (0, 5000)):
+        with pytest.raises(B.DipacoError) as e:
+            B.dipaco_set_work_items(ctx, *bad)
+        assert e.value.status == B.DIPACO_EINVAL
+    for good in (-1, 0, 1, 16):
+        B.dipaco_set_host_threads(ctx, good)
+    for bad in (-2, 1000):
+        with pytest.raises(B.DipacoError):
+            B.dipaco_set_host_threads(ctx, bad)
+    for good in (0, 1 << 20, 1 << 33):
+        B.dipaco_set_host_unit_bytes(ctx, good)
+    with pytest.raises(B.DipacoError):
+        B.dipaco_set_host_unit_bytes(ctx, -5)
+    # the diagnostic needs a device
+    with pytest.raises(B.DipacoError) as e:
+        B.dipaco_selftest_wait_expiry(ctx, 1000, stream=0)
+    assert e.value.status == B.DIPACO_ENODEV
+    B.dipaco_destroy(ctx)
+
+
 def test_compact_shard_contexts_tile_the_problem_exactly_once():
     """dipaco_plan_shard / dipaco_create_shard (Section 3.3, sharded executor): over the shards
     every element of every level is owned exactly once, a shard context is the same grid with the
