@@ -7,6 +7,7 @@
 #endif
 #include <condition_variable>
 #include <cstring>
+#include <exception>
 #include <mutex>
 #include <new>
 #include <thread>
@@ -996,6 +997,8 @@ int dipaco_outer_sync_host(dipaco_ctx *ctx, float *theta_host, float *momentum_h
                               static_cast<cudaStream_t>(cuda_stream));
     } catch (const std::bad_alloc &) {
         return DIPACO_ENOMEM;
+    } catch (const std::exception &) {
+        return DIPACO_ENOMEM;  // the host threads could not be created: a resource limit
     }
 }
 

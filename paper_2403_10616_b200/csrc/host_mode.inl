@@ -69,17 +69,14 @@ public:
     };
     explicit ReplicatePool(int threads)
     {
-        for (int t = 0; t < threads; ++t) workers_.emplace_back([this, t, threads] { work(t, threads); });
-    }
-    ~ReplicatePool()
-    {
-        {
-            std::lock_guard<std::mutex> lock(mutex_);
-            stop_ = true;
+        try {
+            for (int t = 0; t < threads; ++t) workers_.emplace_back([this, t, threads] { work(t, threads); });
+        } catch (...) {
+            shut_down();  // a thread could not be created: end the ones that were, then report
+            throw;
         }
-        wake_.notify_all();
-        for (std::thread &w : workers_) w.join();
     }
+    ~ReplicatePool() { shut_down(); }
     int size() const { return (int)workers_.size(); }
     void run(const Job &job)
     {
@@ -93,6 +90,16 @@ public:
     }
 
 private:
+    void shut_down()
+    {
+        {
+            std::lock_guard<std::mutex> lock(mutex_);
+            stop_ = true;
+        }
+        wake_.notify_all();
+        for (std::thread &w : workers_) w.join();
+        workers_.clear();
+    }
     void work(int t, int threads)
     {
         unsigned long long seen = 0;
