@@ -39,7 +39,7 @@ REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the referen
 # digest is checked and "traffic" is null after any change to them.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9918
 NCU_CAPTURE_SOURCES = ("kernels.cuh", "dipaco.cu", "plan.hpp")
-NCU_CAPTURE_SOURCES_SHA256 = "5d6c0146077d8e204bfa4593d70e9841a12820d60366dba880852f9dcec57db3"
+NCU_CAPTURE_SOURCES_SHA256 = "54666308d163d3de406f885bc824c1a6daea8cc1cc2660b7d84eda34402990a0"
 NCU_CAPTURE_COMMAND = ("ncu --set full --clock-control none -k regex:sync_bulk_kernel -s 3 -c 3 "
                        "python bench.py --level-numel 2000000 --steps 3 --warmup 3 --no-e2e "
                        "--no-chunked --no-cpu-baseline --no-variants --no-other-workloads")
