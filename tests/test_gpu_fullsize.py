@@ -59,7 +59,7 @@ class Sampler:
     """Sampled element indices of every level, and the gathers that turn the full problem into
     the small problem the oracle is run on (same grid, level sizes = number of samples)."""
 
-    def __init__(self, problem, seed=1234):
+    def __init__(self, problem, seed=1234, windows=()):
         cfg = problem.cfg
         gen = torch.Generator(device=DEV)
         gen.manual_seed(seed)
@@ -67,9 +67,11 @@ class Sampler:
         self.idx = []
         for n in cfg.level_numel:
             edge = min(65536, n)
-            self.idx.append(torch.cat([torch.arange(0, edge, device=DEV),
-                                       torch.arange(n - edge, n, device=DEV),
-                                       torch.randint(0, n, (1 << 20,), device=DEV, generator=gen)]))
+            parts = [torch.arange(0, edge, device=DEV), torch.arange(n - edge, n, device=DEV),
+                     torch.randint(0, n, (1 << 20,), device=DEV, generator=gen)]
+            # extra windows of consecutive indices (clipped to the level), e.g. around 2^31
+            parts.extend(torch.arange(max(a, 0), min(b, n), device=DEV) for a, b in windows if a < n)
+            self.idx.append(torch.cat(parts))
         self.small = cfg.scaled(tuple(int(i.numel()) for i in self.idx))
         self.mod_off = problem.module_offsets()
         self.lvl_off = problem.level_offsets()
@@ -206,3 +208,49 @@ def test_host_buffer_entry_point_at_scale_matches_the_oracle_and_the_resident_re
     sampler.check(theta_h, mom_h, rows, want)
     theta_d, mom_d, paths_d = theta_h.to(DEV), mom_h.to(DEV), paths_h.to(DEV)
     assert checksums(theta_d, mom_d, [paths_d[i] for i in range(cfg.num_paths)]) == resident
+
+
+@pytest.mark.parametrize("kernel", ["auto", "vector"])
+def test_a_module_with_more_than_2_pow_31_parameters(kernel):
+    """The largest sizes: one module of 2^31 + 12,293 parameters shared by two paths (bf16), next
+    to a level of two small modules.  Element indices, byte offsets into the copies (4.3 GB each)
+    and the partial-sum scratch all pass 2^31 and 2^32; the module's last five parameters do not
+    fill a 16-byte unit, so the one-element-per-thread kernel runs beyond 2^31 too.  Sampled
+    against the oracle with extra windows on both sides of 2^31 and of 2^32 bytes; the chunk walk
+    (one path per chunk, so the big module carries a partial sum) must give bitwise the same."""
+    big = (1 << 31) + 3 * 4096 + 5
+    cfg = synth.SyncConfig("one-huge-module", (1, 2), (big, 4099), "bf16", weights="tokens",
+                           momentum_std=1e-4)
+    need = cfg.path_params * 2 + 8 * cfg.module_params
+    # the generator holds two fp32 temporaries of the module's size besides the problem itself
+    if free_device_memory() < need + 3 * 4 * big + 8e9:
+        pytest.skip("needs %.0f GB of free device memory" % ((need + 12 * big) / 1e9))
+    code = {"auto": B.DIPACO_KERNEL_AUTO, "vector": B.DIPACO_KERNEL_VECTOR}[kernel]
+
+    def run(problem, chunk_paths):
+        sync = B.OuterSync.for_problem(problem, chunk_paths=chunk_paths)
+        B.dipaco_set_kernel(sync.ctx, code)
+        sync.sync(problem.theta, problem.momentum, problem.paths, problem.reported)
+        assert sync.status() == B.DIPACO_OK
+        sync.close()
+        torch.cuda.synchronize()
+
+    pr = synth.make_problem(cfg, DEV)
+    free_device_memory()
+    half = 1 << 30   # element whose byte offset inside a bf16 copy is 2^31; fp32 offset 2^32
+    sampler = Sampler(pr, windows=[(half - 8192, half + 8192), ((1 << 31) - 8192, big)])
+    before = sampler.inputs(pr)
+    run(pr, 0)
+    want = sampler.expected(pr, before)
+    sampler.check(pr.theta, pr.momentum, pr.paths, want, every=1)
+    assert_every_copy_is_the_cast_of_its_module(pr)
+    first = checksums(pr.theta, pr.momentum, pr.paths)
+    del pr
+    free_device_memory()
+
+    chunked = synth.make_problem(cfg, DEV)
+    free_device_memory()
+    run(chunked, 1)
+    assert checksums(chunked.theta, chunked.momentum, chunked.paths) == first
+    del chunked
+    free_device_memory()
