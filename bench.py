@@ -622,6 +622,27 @@ def run_other_workloads(args, skip_name, tune, local, peak):
         sampler.mark_end()
         clocks = sampler.stop()
         ms = a.elapsed_time(b) / steps
+        graph_us = None
+        if need < 126e6:
+            # launch-bound: the same repeated call (it reuses the kept plan, so it only launches)
+            # captured 100 times in a CUDA graph and replayed
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                h = int(torch.cuda.current_stream().cuda_stream)
+                for _ in range(100):
+                    B.dipaco_outer_sync(ctx, th, mo, arr, problem.reported, h)
+            replays = max(steps // 100, 10)
+            graph.replay()
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(replays):
+                graph.replay()
+            b.record()
+            torch.cuda.synchronize()
+            graph_us = a.elapsed_time(b) / (replays * 100) * 1e3
+            del graph
         ok = B.dipaco_device_status(ctx) == B.DIPACO_OK
         B.dipaco_destroy(ctx)
         alg = synth.algorithmic_bytes(cfg, problem.reported)
@@ -630,6 +651,7 @@ def run_other_workloads(args, skip_name, tune, local, peak):
                  "algorithmic_bytes": alg, "clocks": clocks}
         if need < 126e6:
             entry["us_per_call"] = ms * 1e3
+            entry["us_per_call_cuda_graph"] = graph_us
             entry["note"] = "fits in L2: launch latency, not a roofline point"
         else:
             gbs = alg / (ms * 1e-3) / 1e9

@@ -108,7 +108,12 @@ int dipaco_create(dipaco_ctx **out, int32_t num_levels, const int32_t *modules_p
  * ascending order over the same device pointers, one launch per chunk, carrying fp32 partial
  * sums; the launch that sees a module's last reporting path finishes the module and writes
  * cast(theta') into all of its paths.  A call with the same settings, buffers and mask as the
- * previous one on this context reuses that call's plan and device tables.
+ * previous one on this context reuses that call's plan and device tables: it only launches
+ * kernels (no upload, no allocation, no synchronisation), so it may be recorded in a CUDA graph
+ * by stream capture once one ordinary call has planned it.  Replaying the graph is then the
+ * cheapest way to repeat a small synchronisation (2x2 grid: 5.5 us per replayed call against
+ * 8.2 us per launched call).  Any dipaco_set_* call, another mask or other buffers make the next
+ * call plan and upload again, which must not happen during capture.
  */
 int dipaco_outer_sync(dipaco_ctx *ctx, float *theta, float *momentum, void *const *path_ptrs,
                       const uint8_t *reported, void *cuda_stream);

@@ -683,6 +683,58 @@ def test_a_repeated_call_reuses_its_plan_and_any_change_replans():
     B.dipaco_destroy(ctx)
 
 
+@pytest.mark.parametrize("chunk", [0, 32])
+def test_a_repeated_call_replayed_from_a_cuda_graph_follows_the_oracle(chunk):
+    """A call that reuses the plan of the previous one only launches kernels (no upload, no
+    allocation, no synchronisation), so it can be captured in a CUDA graph.  One replay on the
+    original inputs matches the oracle; three replays give bitwise the result of three calls
+    launched directly.  The ragged last level also puts the tail kernel in the graph."""
+    cfg = synth.CONFIGS["grid16x16-masked"].scaled((2 * 4096 + 72, 4096 + 8, 4096 + 1003))
+    pr = synth.make_problem(cfg, DEV)
+    before = host_state(clone_problem(pr))
+    direct = clone_problem(pr)
+    ctx = make_ctx(pr, chunk)
+    for _ in range(3):
+        B.dipaco_outer_sync(ctx, direct[0].data_ptr(), direct[1].data_ptr(),
+                            [p.data_ptr() for p in direct[2]], pr.reported)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    B.dipaco_destroy(ctx)
+
+    state = clone_problem(pr)
+    ptrs = B.ptr_array([p.data_ptr() for p in state[2]])
+    ctx = make_ctx(pr, chunk)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    # the call that plans and uploads the tables stays outside the graph
+    B.dipaco_outer_sync(ctx, state[0].data_ptr(), state[1].data_ptr(), ptrs, pr.reported, stream=stream)
+    stream.synchronize()
+    launches_planned = B.dipaco_launch_count(ctx)
+    assert launches_planned >= 2
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        B.dipaco_outer_sync(ctx, state[0].data_ptr(), state[1].data_ptr(), ptrs, pr.reported,
+                            stream=torch.cuda.current_stream())
+    assert B.dipaco_launch_count(ctx) == 2 * launches_planned
+
+    def restore():
+        state[0].copy_(pr.theta); state[1].copy_(pr.momentum)
+        for p, q in zip(state[2], pr.paths):
+            p.copy_(q)
+        torch.cuda.synchronize()
+
+    restore()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert_matches_oracle(pr, before, state)
+    restore()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert_states_bitwise_equal(state, direct)
+    assert B.dipaco_device_status(ctx) == B.DIPACO_OK
+    B.dipaco_destroy(ctx)
+
+
 def test_a_wait_that_runs_out_is_reported_once_and_the_context_recovers():
     """The time-out path end to end, without disturbing the pipeline kernels: the diagnostic
     entry point makes one bounded wait (1 ms) run out on a barrier nothing completes.  The kernel
