@@ -579,10 +579,14 @@ def run_other_workloads(args, skip_name, tune, local, peak):
     from paper_2403_10616_b200 import binding as B
     from paper_2403_10616_b200 import synth
     out = []
-    for name in ("grid2x2", "grid4x4", "grid16x16-masked", "grid4x4x4x4"):
+    # the last entry is the 16x16 grid with an odd level size: every module of theta and every slot
+    # of every path copy then starts inside a 16-byte unit (rows of one block: all eight positions),
+    # so the bulk-copy kernel cannot take it and the shifted vector kernel does
+    odd = synth.CONFIGS["grid16x16"].scaled((20_000_003,) * 3, name="grid16x16-odd-level-size")
+    for name in ("grid2x2", "grid4x4", "grid16x16-masked", "grid4x4x4x4", odd.name):
         if name == skip_name:
             continue
-        cfg = synth.CONFIGS[name]
+        cfg = odd if name == odd.name else synth.CONFIGS[name]
         es = 2 if cfg.path_dtype == "bf16" else 4
         need = cfg.path_params * es + 8 * cfg.module_params
         torch.cuda.empty_cache()
@@ -657,6 +661,9 @@ def run_other_workloads(args, skip_name, tune, local, peak):
             gbs = alg / (ms * 1e-3) / 1e9
             entry.update({"algorithmic_gbs": gbs, "frac_of_peak": gbs / peak,
                           "frac_of_nominal_8tbs": gbs / 8000.0})
+            if name == odd.name:
+                entry["level_numel"] = list(cfg.level_numel)
+                entry["kernel"] = "sync_direct_kernel<.,8,shifted> (buffers at odd element offsets)"
         out.append(entry)
         del problem, arr
         torch.cuda.empty_cache()

@@ -24,7 +24,8 @@ constexpr int STAGING_SLOTS = 4;
 constexpr size_t SMEM_LIMIT = 227 * 1024;  // opt-in dynamic shared memory per CTA on sm_100
 constexpr size_t SMEM_PER_SM = 228 * 1024;
 constexpr size_t SMEM_CTA_RESERVE = 1024;  // per-CTA reservation the driver adds
-constexpr int64_t RAGGED_TILE = 1024;      // split granularity of the scalar kernel
+constexpr int64_t RAGGED_TILE = 256;       // split granularity of the scalar kernel: one element per thread
+constexpr int64_t SHIFT_TILE = 2048;       // 256 threads * 8 elements: one CTA step of the shifted vector kernel
 constexpr int MAX_COUNTERS = 256;          // work counters (one per bulk launch of an upload)
 
 enum SyncState { STATE_IDLE = 0, STATE_ACCUMULATING = 1 };
@@ -40,7 +41,8 @@ struct Staging {
 struct PackedLaunch {
     size_t passes_off = 0, contribs_off = 0, members_off = 0;
     size_t bulk_segs_off = 0, bulk_first_off = 0, rag_segs_off = 0, rag_first_off = 0;
-    int bulk_ctas = 0, rag_ctas = 0;
+    size_t shv_segs_off = 0, shv_first_off = 0;  // ranges of the shifted vector kernel (misaligned modules)
+    int bulk_ctas = 0, rag_ctas = 0, shv_ctas = 0;
     int io_arrays = 2;
     int units = 2;                        // 16-byte units per compute thread and tile of this launch
     bool aligned_kernel_is_vector = false;
@@ -229,7 +231,17 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     std::vector<ContribDev> contribs;
     std::vector<void *> members;
     std::vector<int64_t> bulk_begin(specs.size(), 0), bulk_end(specs.size(), 0);
-    std::vector<int64_t> rag_begin(specs.size(), 0), rag_end(specs.size(), 0);
+    std::vector<int64_t> shv_begin(specs.size(), 0), shv_end(specs.size(), 0);
+    // ranges of the one-element-per-thread kernel: a pass can have one before and one after its
+    // vector range
+    std::vector<int32_t> rag_pass;
+    std::vector<int64_t> rag_begin, rag_end;
+    auto add_ragged = [&](size_t pass, int64_t b, int64_t e) {
+        if (b >= e) return;
+        rag_pass.push_back((int32_t)pass);
+        rag_begin.push_back(b);
+        rag_end.push_back(e);
+    };
     bool any_partial = false;
     for (const PassSpec &sp : specs)
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
@@ -257,9 +269,18 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (((sp.flags & PASS_CAST_IN) || sp.cast_out) && !ctx->cast_scratch) return DIPACO_ESTATE;
         bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
                        ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
+        // the fp32 arrays all start at the same place within a 16-byte unit: a range can be cut
+        // so that every thread's first element is 16-byte aligned in all of them at once
+        const uintptr_t state_rem = (uintptr_t)(theta + m.theta_off) % 16;
+        bool state_congruent = (uintptr_t)(momentum + m.theta_off) % 16 == state_rem;
         if (ctx->optimizer == DIPACO_OPT_ADAM) {
             const float *v = ctx->second_moment_staged ? ctx->second_moment_staged : ctx->second_moment;
             aligned = aligned && ((uintptr_t)(v + m.theta_off) % 16 == 0);
+            state_congruent = state_congruent && (uintptr_t)(v + m.theta_off) % 16 == state_rem;
+        }
+        if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) {
+            aligned = aligned && ((uintptr_t)(ctx->partial + m.partial_off) % 16 == 0);
+            state_congruent = state_congruent && (uintptr_t)(ctx->partial + m.partial_off) % 16 == state_rem;
         }
         pd.contrib_begin = (int)contribs.size();
         for (size_t j = 0; j < sp.contributors.size(); ++j) {
@@ -289,6 +310,13 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
                 members.push_back(dst);
             }
         pd.member_count = (int)members.size() - pd.member_begin;
+        // destinations with the same position inside a 16-byte unit next to each other: the
+        // shifted vector kernel rebuilds its realigned units only when that position changes
+        // (the order of the destinations has no effect on the result)
+        if (!aligned)
+            std::stable_sort(members.begin() + pd.member_begin, members.end(), [](void *x, void *y) {
+                return ((uintptr_t)x & 15u) < ((uintptr_t)y & 15u);
+            });
 
         // The vector kernel takes full tiles; the bulk-copy kernel also takes a partial last tile
         // as long as it is a whole number of 16-byte units of path data.
@@ -302,22 +330,41 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (aligned && ctx->kernel == DIPACO_KERNEL_VECTOR) full = (hi - lo) / tile * tile;
         if (aligned && ctx->kernel == DIPACO_KERNEL_AUTO) full = (hi - lo) / unit * unit;
         bulk_begin[i] = lo; bulk_end[i] = lo + full;
-        rag_begin[i] = lo + full; rag_end[i] = hi;
+        if (!aligned && state_congruent && ctx->kernel != DIPACO_KERNEL_SCALAR) {
+            // Path buffers at odd element offsets (or a range that starts inside a 16-byte unit):
+            // the shifted vector kernel takes whole steps from the first element at which theta
+            // is 16-byte aligned.  It reads the aligned 16-byte units around each thread's data,
+            // so the last 8 elements of the range stay with the one-element kernel: no load
+            // reaches past the module's slot in a path buffer.
+            const uintptr_t rem = (state_rem + (uintptr_t)(lo % 4) * 4) % 16;
+            const int64_t first = lo + (int64_t)((16 - rem) % 16) / 4;
+            const int64_t steps = hi - 8 > first ? (hi - 8 - first) / SHIFT_TILE : 0;
+            if (steps > 0) {
+                shv_begin[i] = first;
+                shv_end[i] = first + steps * SHIFT_TILE;
+                add_ragged(i, lo, first);
+                add_ragged(i, shv_end[i], hi);
+                continue;
+            }
+        }
+        add_ragged(i, lo + full, hi);
     }
 
-    std::vector<Segment> bulk_segs, rag_segs;
-    std::vector<int32_t> bulk_first, rag_first;
+    std::vector<Segment> bulk_segs, rag_segs, shv_segs;
+    std::vector<int32_t> bulk_first, rag_first, shv_first;
     const bool vector_kernel = ctx->kernel == DIPACO_KERNEL_VECTOR;
     int bulk_ctas = ctx->sm_count * (vector_kernel ? 8 : ctx->ctas_per_sm);
-    int64_t bulk_tiles = 0, rag_tiles = 0;
+    int64_t bulk_tiles = 0, rag_tiles = 0, shv_tiles = 0;
     double bulk_bytes = 0.0, contrib_elems = 0.0, bulk_elems = 0.0;
     for (size_t i = 0; i < specs.size(); ++i) {
         contrib_elems += (double)specs[i].contributors.size() * (double)(bulk_end[i] - bulk_begin[i]);
         bulk_elems += (double)(bulk_end[i] - bulk_begin[i]);
         bulk_tiles += (bulk_end[i] - bulk_begin[i] + tile - 1) / tile;
         bulk_bytes += pass_cost_per_elem(specs[i], es) * (double)(bulk_end[i] - bulk_begin[i]);
-        rag_tiles += (rag_end[i] - rag_begin[i] + RAGGED_TILE - 1) / RAGGED_TILE;
+        shv_tiles += (shv_end[i] - shv_begin[i]) / SHIFT_TILE;
     }
+    for (size_t r = 0; r < rag_begin.size(); ++r)
+        rag_tiles += (rag_end[r] - rag_begin[r] + RAGGED_TILE - 1) / RAGGED_TILE;
     if (bulk_tiles < bulk_ctas) bulk_ctas = (int)bulk_tiles;
     int rag_ctas = (int)std::min<int64_t>(rag_tiles, (int64_t)ctx->sm_count * 8);
     int64_t total_items = 0;
@@ -344,7 +391,10 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (total_items < bulk_ctas) bulk_ctas = (int)total_items;
     }
     if (rag_ctas > 0)
-        split_segments(specs, rag_begin, rag_end, es, RAGGED_TILE, rag_ctas, rag_segs, rag_first);
+        split_segments(specs, rag_begin, rag_end, es, RAGGED_TILE, rag_ctas, rag_segs, rag_first, &rag_pass);
+    const int shv_ctas = (int)std::min<int64_t>(shv_tiles, (int64_t)ctx->sm_count * 8);
+    if (shv_ctas > 0)
+        split_segments(specs, shv_begin, shv_end, es, SHIFT_TILE, shv_ctas, shv_segs, shv_first);
 
     auto append = [&](const void *src, size_t bytes) -> size_t {
         const size_t off = align_up(blob.size(), 16);
@@ -360,8 +410,11 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     out.bulk_first_off = append(bulk_first.data(), bulk_first.size() * sizeof(int32_t));
     out.rag_segs_off = append(rag_segs.data(), rag_segs.size() * sizeof(Segment));
     out.rag_first_off = append(rag_first.data(), rag_first.size() * sizeof(int32_t));
+    out.shv_segs_off = append(shv_segs.data(), shv_segs.size() * sizeof(Segment));
+    out.shv_first_off = append(shv_first.data(), shv_first.size() * sizeof(int32_t));
     out.bulk_ctas = bulk_ctas;
     out.rag_ctas = rag_ctas;
+    out.shv_ctas = shv_ctas;
     out.io_arrays = io_arrays;
     out.units = units;
     out.aligned_kernel_is_vector = vector_kernel;
@@ -505,6 +558,16 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
             rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, pl.units, pl.mean_contributors, stream);
         }
         if (rc != DIPACO_OK) return rc;
+        ++ctx->launches;
+    }
+    if (pl.shv_ctas > 0) {
+        lp.segs = reinterpret_cast<const SegmentDev *>(base + pl.shv_segs_off);
+        lp.cta_first = reinterpret_cast<const int *>(base + pl.shv_first_off);
+        if (ctx->dtype == DIPACO_BF16)
+            sync_direct_kernel<__nv_bfloat16, 8, true><<<pl.shv_ctas, 256, 0, stream>>>(lp);
+        else
+            sync_direct_kernel<float, 8, true><<<pl.shv_ctas, 256, 0, stream>>>(lp);
+        if (cudaGetLastError() != cudaSuccess) return DIPACO_ECUDA;
         ++ctx->launches;
     }
     if (pl.rag_ctas > 0) {

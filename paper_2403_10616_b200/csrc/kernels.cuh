@@ -4,6 +4,9 @@
 // give bitwise identical results:
 //   sync_direct_kernel<PathT,1>   one element per thread, any alignment (ragged tails, odd offsets)
 //   sync_direct_kernel<PathT,8>   128-bit register loads/stores on 16-byte aligned full tiles
+//   sync_direct_kernel<PathT,8,true>  the same for path buffers at any element alignment, each
+//                                 with its own: 128-bit accesses to the aligned units around the
+//                                 data, funnel shifts, and a warp shuffle to realign the stores
 //   sync_bulk_kernel<PathT,NU>    persistent, warp-specialised: a scheduler warp draws work items
 //                                 from a counter, one warp streams tiles into a shared-memory
 //                                 ring with bulk async copies (TMA, 1-D), eight warps reduce and
@@ -186,11 +189,94 @@ template <> struct Unit<__nv_bfloat16> {
 };
 
 // ------------------------------------------------------------------------------------------
+// Path data that is only element-aligned.  A thread's 16 bytes then straddle two aligned 16-byte
+// units; both are loaded whole and the wanted bytes are cut out with funnel shifts.
+
+// The 16 bytes that start s bytes into the 32 bytes (lo, hi); s even, 0 <= s < 16.  Branch free (a
+// word-granular barrel shift by selects, then one funnel shift by 0 or 16 bits), so that the
+// compiler can keep the loads of several contributors in flight across it.
+__device__ __forceinline__ uint4 cut16(const uint4 &lo, const uint4 &hi, unsigned s)
+{
+    const bool by1 = (s & 4u) != 0, by2 = (s & 8u) != 0;
+    const unsigned r = (s & 2u) * 8u;
+    const unsigned w0 = lo.x, w1 = lo.y, w2 = lo.z, w3 = lo.w, w4 = hi.x, w5 = hi.y, w6 = hi.z, w7 = hi.w;
+    const unsigned x0 = by1 ? w1 : w0, x1 = by1 ? w2 : w1, x2 = by1 ? w3 : w2, x3 = by1 ? w4 : w3,
+                   x4 = by1 ? w5 : w4, x5 = by1 ? w6 : w5, x6 = by1 ? w7 : w6;
+    const unsigned y0 = by2 ? x2 : x0, y1 = by2 ? x3 : x1, y2 = by2 ? x4 : x2, y3 = by2 ? x5 : x3,
+                   y4 = by2 ? x6 : x4;
+    return make_uint4(__funnelshift_r(y0, y1, r), __funnelshift_r(y1, y2, r), __funnelshift_r(y2, y3, r),
+                      __funnelshift_r(y3, y4, r));
+}
+
+// UNITS * 16 bytes from an address that is only element-aligned: the aligned 16-byte units that
+// contain them (one more than UNITS when the address lies inside a unit) and how far into the
+// first unit the data starts.  Up to 15 bytes before and after the wanted range are read, inside
+// the same aligned units.  Loading and cutting are separate so that a caller can issue the loads of
+// several sources before it uses any of them.
+template <int UNITS>
+__device__ __forceinline__ unsigned load_around(const void *p, uint4 *raw)
+{
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p);
+    const unsigned s = (unsigned)(a & 15u);
+    const uint4 *base = reinterpret_cast<const uint4 *>(a - s);
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) raw[u] = __ldcs(base + u);
+    raw[UNITS] = make_uint4(0u, 0u, 0u, 0u);
+    if (s != 0) raw[UNITS] = __ldcs(base + UNITS);
+    return s;
+}
+
+__device__ __forceinline__ uint4 shfl_down1(const uint4 &v)
+{
+    return make_uint4(__shfl_down_sync(0xffffffffu, v.x, 1), __shfl_down_sync(0xffffffffu, v.y, 1),
+                      __shfl_down_sync(0xffffffffu, v.z, 1), __shfl_down_sync(0xffffffffu, v.w, 1));
+}
+
+__device__ __forceinline__ unsigned word_at(const uint4 &v, int i)
+{
+    return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+}
+
+// Element i (of the 16-byte unit v) to *dst.
+__device__ __forceinline__ void store_element(float *dst, const uint4 &v, int i)
+{
+    __stcs(reinterpret_cast<unsigned *>(dst), word_at(v, i));
+}
+__device__ __forceinline__ void store_element(__nv_bfloat16 *dst, const uint4 &v, int i)
+{
+    const unsigned w = word_at(v, i >> 1);
+    __stcs(reinterpret_cast<unsigned short *>(dst), (unsigned short)((i & 1) ? (w >> 16) : (w & 0xffffu)));
+}
+
+// The bytes of a CTA's step that do not fill an aligned 16-byte unit of a shifted destination: the
+// first `count` elements of the step's first thread (from_end = false) or the last `count` elements
+// of its last thread (from_end = true).  `unit` is that thread's first, or last, 16 bytes.
+template <typename PathT>
+__device__ __forceinline__ void store_edge_elements(PathT *first_or_last, const uint4 &unit, int count,
+                                                    bool from_end)
+{
+    constexpr int PER = 16 / (int)sizeof(PathT);  // elements per 16 bytes
+#pragma unroll
+    for (int i = 0; i < PER - 1; ++i) {
+        if (i < count) {
+            if (from_end) store_element(first_or_last - i, unit, PER - 1 - i);
+            else store_element(first_or_last + i, unit, i);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Direct kernels: every thread owns VEC consecutive elements and walks the contributors itself.
 
-template <typename PathT, int VEC>
-__global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
+// SHIFTED (VEC = 8 only): theta, momentum, partial sums and second moment are 16-byte aligned at
+// every thread's first element (the host cuts the range that way); the path buffers and the cast
+// scratch may sit at any element alignment, each its own.  A thread loads the aligned 16-byte
+// units around its data and cuts its bytes out; stores are put together into aligned units again
+// across neighbouring threads.  Segments are whole CTA steps of 2048 elements.
+template <typename PathT, int VEC, bool SHIFTED = false>
+__global__ void __launch_bounds__(256, SHIFTED ? 2 : 0) sync_direct_kernel(LaunchParams p)
 {
+    static_assert(!SHIFTED || VEC == 8, "the shifted variant is the 8-element one");
     // a context whose error word is set (a bounded wait ran out earlier) does no further work
     // until the host has read the status
     if (*reinterpret_cast<volatile const int *>(p.error_word) != 0) return;
@@ -234,11 +320,21 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
             } else {
                 constexpr int UE = Unit<PathT>::UE;
                 constexpr int UNITS = VEC / UE;  // 16-byte loads per contributor
-                constexpr int BATCH = 8 / UNITS; // contributors whose loads are issued together
+                // contributors whose loads are issued together (the shifted variant loads one
+                // more unit per contributor: 48 registers of path data in flight either way)
+                constexpr int BATCH = SHIFTED ? (UNITS == 1 ? 6 : 3) : 8 / UNITS;
                 if (pass.flags & KPASS_CAST_IN) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(cast_src + k);
+                    if constexpr (SHIFTED) {
+                        uint4 around[UNITS + 1];
+                        const unsigned shift = load_around<UNITS>(cast_src + k, around);
 #pragma unroll
-                    for (int u = 0; u < UNITS; ++u) Unit<PathT>::widen(__ldcs(src + u), th + u * UE);
+                        for (int u = 0; u < UNITS; ++u)
+                            Unit<PathT>::widen(cut16(around[u], around[u + 1], shift), th + u * UE);
+                    } else {
+                        const uint4 *src = reinterpret_cast<const uint4 *>(cast_src + k);
+#pragma unroll
+                        for (int u = 0; u < UNITS; ++u) Unit<PathT>::widen(__ldcs(src + u), th + u * UE);
+                    }
                 } else {
 #pragma unroll
                     for (int v = 0; v < VEC; v += 4) {
@@ -257,17 +353,23 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
                     for (int v = 0; v < VEC; ++v) acc[v] = 0.0f;
                 }
                 for (int j0 = 0; j0 < pass.contrib_count; j0 += BATCH) {
-                    uint4 raw[BATCH][UNITS];
+                    uint4 raw[BATCH][UNITS + (SHIFTED ? 1 : 0)];
+                    unsigned shift[BATCH];  // SHIFTED: how far into raw[b][0] the data starts
                     float coeff[BATCH];
 #pragma unroll
                     for (int b = 0; b < BATCH; ++b) {
+                        shift[b] = 0;
                         if (j0 + b < pass.contrib_count) {
                             const ContribDev c = contribs[j0 + b];
                             coeff[b] = c.coeff;
-                            const uint4 *src = reinterpret_cast<const uint4 *>(
-                                static_cast<const PathT *>(c.src) + k);
+                            if constexpr (SHIFTED) {
+                                shift[b] = load_around<UNITS>(static_cast<const PathT *>(c.src) + k, raw[b]);
+                            } else {
+                                const uint4 *src = reinterpret_cast<const uint4 *>(
+                                    static_cast<const PathT *>(c.src) + k);
 #pragma unroll
-                            for (int u = 0; u < UNITS; ++u) raw[b][u] = __ldcs(src + u);
+                                for (int u = 0; u < UNITS; ++u) raw[b][u] = __ldcs(src + u);
+                            }
                         }
                     }
 #pragma unroll
@@ -276,7 +378,10 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
 #pragma unroll
                             for (int u = 0; u < UNITS; ++u) {
                                 float x[UE];
-                                Unit<PathT>::widen(raw[b][u], x);
+                                if constexpr (SHIFTED)
+                                    Unit<PathT>::widen(cut16(raw[b][u], raw[b][u + 1], shift[b]), x);
+                                else
+                                    Unit<PathT>::widen(raw[b][u], x);
 #pragma unroll
                                 for (int i = 0; i < UE; ++i)
                                     acc[u * UE + i] =
@@ -347,10 +452,58 @@ __global__ void __launch_bounds__(256) sync_direct_kernel(LaunchParams p)
                     uint4 out[UNITS];
 #pragma unroll
                     for (int u = 0; u < UNITS; ++u) out[u] = Unit<PathT>::narrow(th + u * UE);
-                    for (int j = 0; j < pass.member_count; ++j) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(static_cast<PathT *>(members[j]) + k);
+                    if constexpr (SHIFTED) {
+                        // A destination that sits sh bytes into a 16-byte unit is written in
+                        // aligned units all the same: the unit that straddles two threads takes
+                        // its first sh bytes from the end of the earlier thread's data and the
+                        // rest from the start of the next thread's (next lane by shuffle, next
+                        // warp through shared memory).  That unit reaches into bytes that the
+                        // next thread reads as input: inside a warp all lanes have their inputs
+                        // by now, and the barrier makes it so across the warps of the CTA.  Only
+                        // the two ends of the CTA's 2048 elements are left over and go out
+                        // element by element.  The host sorts the members of a pass by their
+                        // shift, so the realigned units are rebuilt once per shift.
+                        __shared__ uint4 first_unit[8];
+                        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+                        uint4 next_first = shfl_down1(out[0]);
+                        if (lane == 0) first_unit[warp] = out[0];
+                        __syncthreads();
+                        if (lane == 31 && warp < 7) next_first = first_unit[warp + 1];
+                        __syncthreads();
+                        const bool last_thread = threadIdx.x == 255;
+                        unsigned current = 0;
+                        uint4 realigned[UNITS];
+                        for (int j = 0; j < pass.member_count; ++j) {
+                            PathT *dst = static_cast<PathT *>(members[j]) + k;
+                            const uintptr_t a = reinterpret_cast<uintptr_t>(dst);
+                            const unsigned sh = (unsigned)(a & 15u);
+                            if (sh == 0) {
+                                uint4 *d16 = reinterpret_cast<uint4 *>(dst);
 #pragma unroll
-                        for (int u = 0; u < UNITS; ++u) __stcs(dst + u, out[u]);
+                                for (int u = 0; u < UNITS; ++u) __stcs(d16 + u, out[u]);
+                                continue;
+                            }
+                            if (sh != current) {
+                                current = sh;
+#pragma unroll
+                                for (int u = 0; u < UNITS; ++u)
+                                    realigned[u] = cut16(out[u], u + 1 < UNITS ? out[u + 1] : next_first, 16u - sh);
+                            }
+                            uint4 *d16 = reinterpret_cast<uint4 *>(a + 16u - sh);
+#pragma unroll
+                            for (int u = 0; u + 1 < UNITS; ++u) __stcs(d16 + u, realigned[u]);
+                            if (!last_thread) __stcs(d16 + UNITS - 1, realigned[UNITS - 1]);
+                            if (threadIdx.x == 0)
+                                store_edge_elements<PathT>(dst, out[0], (int)(16u - sh) / (int)sizeof(PathT), false);
+                            if (last_thread)
+                                store_edge_elements<PathT>(dst + VEC - 1, out[UNITS - 1], (int)sh / (int)sizeof(PathT), true);
+                        }
+                    } else {
+                        for (int j = 0; j < pass.member_count; ++j) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(static_cast<PathT *>(members[j]) + k);
+#pragma unroll
+                            for (int u = 0; u < UNITS; ++u) __stcs(dst + u, out[u]);
+                        }
                     }
                 }
             }

@@ -126,9 +126,11 @@ inline bool build_grid(Grid &g, int L, const int32_t *K, const int64_t *N, int P
         m.partial_off = -1;
         if (g.num_chunks > 1 && !m.members.empty() &&
             g.chunk_of(m.members.front()) != g.chunk_of(m.members.back())) {
-            m.partial_off = g.scratch_elems;
-            // keep every module's slab 16-byte aligned for vector / bulk access
-            g.scratch_elems += (m.numel + 3) / 4 * 4;
+            // A module's slab starts where its theta starts within a 16-byte unit (at a multiple
+            // of four elements when theta_off is one), so that vector and bulk accesses that are
+            // aligned for theta are aligned for the partial sum too.
+            m.partial_off = g.scratch_elems + (m.theta_off & 3);
+            g.scratch_elems = (m.partial_off + m.numel + 3) / 4 * 4;
         }
     }
     return true;
@@ -303,15 +305,19 @@ inline double pass_cost_per_elem(const PassSpec &p, int elem_size)
 
 // Split [0, full_tiles*tile) of every pass in `which` over num_ctas CTAs with equal cost, cutting
 // at tile boundaries.  cta_first has num_ctas+1 entries indexing into segs.
+// Range i belongs to pass (*pass_of)[i], or to pass i when pass_of is null (one range per pass).
 inline void split_segments(const std::vector<PassSpec> &passes, const std::vector<int64_t> &begin,
                            const std::vector<int64_t> &end, int elem_size, int64_t tile,
-                           int num_ctas, std::vector<Segment> &segs, std::vector<int32_t> &cta_first)
+                           int num_ctas, std::vector<Segment> &segs, std::vector<int32_t> &cta_first,
+                           const std::vector<int32_t> *pass_of = nullptr)
 {
     segs.clear();
     cta_first.assign((size_t)num_ctas + 1, 0);
+    const size_t ranges = begin.size();
+    auto pass_index = [&](size_t i) -> size_t { return pass_of ? (size_t)(*pass_of)[i] : i; };
     double total = 0.0;
-    for (size_t i = 0; i < passes.size(); ++i)
-        total += pass_cost_per_elem(passes[i], elem_size) * (double)(end[i] - begin[i]);
+    for (size_t i = 0; i < ranges; ++i)
+        total += pass_cost_per_elem(passes[pass_index(i)], elem_size) * (double)(end[i] - begin[i]);
     if (total <= 0.0 || num_ctas < 1) return;
     // CTA b ends at the tile boundary nearest to the cumulative cost (b+1)*share, so rounding
     // does not pile up on the last CTA.  A CTA may end up empty on very small launches.
@@ -319,8 +325,8 @@ inline void split_segments(const std::vector<PassSpec> &passes, const std::vecto
     int cta = 0;
     double cum = 0.0;  // cost of everything handed out so far
     cta_first[0] = 0;
-    for (size_t i = 0; i < passes.size(); ++i) {
-        const double per_tile = pass_cost_per_elem(passes[i], elem_size) * (double)tile;
+    for (size_t i = 0; i < ranges; ++i) {
+        const double per_tile = pass_cost_per_elem(passes[pass_index(i)], elem_size) * (double)tile;
         int64_t pos = begin[i];
         while (pos < end[i]) {
             const int64_t tiles_left = (end[i] - pos + tile - 1) / tile;
@@ -335,7 +341,7 @@ inline void split_segments(const std::vector<PassSpec> &passes, const std::vecto
                 }
             }
             const int64_t stop = std::min(end[i], pos + take * tile);
-            segs.push_back(Segment{(int32_t)i, 0, pos, stop});
+            segs.push_back(Segment{(int32_t)pass_index(i), 0, pos, stop});
             cum += per_tile * (double)take;
             pos = stop;
         }

@@ -140,9 +140,10 @@ def test_random_structure_matches_the_oracle(seed):
         parts = [theta[int(mod_off[l]) + int(table[i, l]) * n:int(mod_off[l]) + (int(table[i, l]) + 1) * n]
                  + torch.empty(n, device=DEV).normal_(0, 1e-3, generator=gen) for l, n in enumerate(numel)]
         row = torch.cat(parts).to(tdt)
-        if opts["misalign"]:                       # element-aligned only
-            back = torch.empty(row.numel() + 4, dtype=tdt, device=DEV)
-            view = back[1:1 + row.numel()]
+        if opts["misalign"]:                       # element-aligned only, every path its own offset
+            back = torch.empty(row.numel() + 8, dtype=tdt, device=DEV)
+            off = 1 + i % 7
+            view = back[off:off + row.numel()]
             view.copy_(row)
             keepalive.append(back)
             row = view

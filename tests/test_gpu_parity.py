@@ -245,7 +245,7 @@ def test_masked_paths_are_not_read_and_nan_propagates():
     assert torch.isnan(state[0]).sum().item() == 1
 
 
-def test_misaligned_path_pointers_take_the_scalar_path():
+def test_misaligned_path_pointers_on_small_modules_take_the_scalar_path():
     cfg = synth.SyncConfig("mis", (1, 2, 2), (4100, 2052, 1000), "bf16", seed=9)
     pr = synth.make_problem(cfg, DEV)
     before = host_state(clone_problem(pr))
@@ -259,6 +259,55 @@ def test_misaligned_path_pointers_take_the_scalar_path():
     state = (pr.theta.clone(), pr.momentum.clone(), paths)
     run_gpu(pr, state)
     assert_matches_oracle(pr, before, state)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("chunk", [0, 4])
+def test_path_buffers_at_any_element_alignment_take_the_shifted_vector_kernel(dtype, chunk):
+    """Every path copy starts at its own element offset within a 16-byte unit (all eight of them
+    for bf16, all four for fp32) and the level sizes are odd, so the modules of theta, the slots
+    inside the copies and the partial sums all start inside 16-byte units.  The vector kernel for
+    shifted buffers takes the bulk of every module, the one-element kernel a few elements before
+    and after: against the oracle, and bitwise equal to the one-element kernel on its own."""
+    cfg = synth.SyncConfig("shifted", (1, 3, 3), (3 * 2048 + 5, 2 * 2048 + 1003, 5 * 2048 + 77), dtype,
+                           weights="tokens", momentum_std=1e-4, seed=9)
+    pr = synth.make_problem(cfg, DEV)
+    before = host_state(clone_problem(pr))
+    per = cfg.params_per_path
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    slots = 16 // (2 if dtype == "bf16" else 4)
+    reported = np.ones(cfg.num_paths, dtype=np.uint8)
+    reported[4] = 0
+
+    def misaligned_state():
+        backing = [torch.empty(per + 16, dtype=tdt, device=DEV) for _ in range(cfg.num_paths)]
+        paths = []
+        for i, b in enumerate(backing):
+            off = i % slots
+            view = b[off:off + per]
+            view.copy_(pr.paths[i])
+            assert view.data_ptr() % 16 == off * view.element_size()
+            paths.append(view)
+        return (pr.theta.clone(), pr.momentum.clone(), paths), backing
+
+    results = {}
+    for kernel in (B.DIPACO_KERNEL_AUTO, B.DIPACO_KERNEL_VECTOR, B.DIPACO_KERNEL_SCALAR):
+        state, backing = misaligned_state()
+        guard = [b.clone() for b in backing]
+        launches = run_gpu(pr, state, reported=reported, chunk_paths=chunk, kernel=kernel)
+        if chunk == 0:
+            # one launch of the one-element kernel alone; with the vector kernel one more
+            assert launches == (1 if kernel == B.DIPACO_KERNEL_SCALAR else 2)
+        assert_matches_oracle(pr, before, state, reported=reported)
+        # nothing outside the copies was written (the stores of aligned units stop at the edges)
+        for i, (b, g) in enumerate(zip(backing, guard)):
+            off = i % slots
+            bits = torch.int16 if dtype == "bf16" else torch.int32
+            assert torch.equal(b[:off].view(bits), g[:off].view(bits))
+            assert torch.equal(b[off + per:].view(bits), g[off + per:].view(bits))
+        results[kernel] = state
+    assert_states_bitwise_equal(results[B.DIPACO_KERNEL_AUTO], results[B.DIPACO_KERNEL_SCALAR])
+    assert_states_bitwise_equal(results[B.DIPACO_KERNEL_VECTOR], results[B.DIPACO_KERNEL_SCALAR])
 
 
 def test_runs_are_bitwise_reproducible():
