@@ -81,6 +81,9 @@ def parse_args():
                          "host-buffer leg (-1 = library default, 0 = none: one download per path)")
     ap.add_argument("--items-per-cta", type=int, default=0)
     ap.add_argument("--item-kb", type=int, default=0)
+    ap.add_argument("--separate-buffers", action="store_true",
+                    help="one allocation per path copy instead of rows of one block (with an odd "
+                         "level size the copies then all sit at the same place within a 16-byte unit)")
     ap.add_argument("--no-other-workloads", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-chunked", action="store_true")
@@ -355,7 +358,7 @@ def run_ours(args):
     if need * 1.02 > free:
         raise SystemExit("workload needs %.1f GB of device memory, %.1f GB free" % (need / 1e9, free / 1e9))
 
-    problem = synth.make_problem(cfg, device)
+    problem = synth.make_problem(cfg, device, separate_buffers=args.separate_buffers)
     torch.cuda.synchronize()
     ptrs = [p.data_ptr() for p in problem.paths]
     kernel = {"auto": B.DIPACO_KERNEL_AUTO, "vector": B.DIPACO_KERNEL_VECTOR,

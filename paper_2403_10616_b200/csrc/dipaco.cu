@@ -46,6 +46,7 @@ struct PackedLaunch {
     int io_arrays = 2;
     int units = 2;                        // 16-byte units per compute thread and tile of this launch
     bool aligned_kernel_is_vector = false;
+    bool shifted = false;                 // some path buffer of a bulk pass sits inside a 16-byte unit
     int num_passes = 0, total_items = 0;  // dynamic scheduling of the bulk-copy kernel
     double mean_contributors = 0.0;       // per element of the bulk range
 };
@@ -97,7 +98,7 @@ struct dipaco_ctx {
     bool cast_scratch_tried = false;
     int *error_word = nullptr;
     int *counters = nullptr;  // MAX_COUNTERS work counters for the bulk-copy kernel
-    bool smem_attr_set[2][3] = {{false, false, false}, {false, false, false}};
+    bool smem_attr_set[2][3][2] = {};  // [path type][units per thread][shifted variant]
 
     // round state of the incremental API
     int state = STATE_IDLE;
@@ -175,22 +176,24 @@ int64_t tile_elems(const dipaco_ctx *ctx)
 }
 
 // Shared memory of one bulk-kernel CTA for a given tile and depth.
-size_t bulk_smem_bytes(const dipaco_ctx *ctx, int units, int stages, int io_arrays, int io_slots)
+size_t bulk_smem_bytes(const dipaco_ctx *ctx, int units, int stages, int io_arrays, int io_slots,
+                       bool shifted = true)
 {
     const size_t tile = (size_t)tile_elems_of(ctx, units);
     const size_t stage = tile * ctx->elem_size;
-    size_t bytes = (size_t)stages * stage + (size_t)io_slots * io_arrays * tile * 4;
+    // (the kernel variant for shifted path buffers loads 16 bytes more into every ring slot)
+    size_t bytes = (size_t)stages * (stage + (shifted ? 16 : 0)) + (size_t)io_slots * io_arrays * tile * 4;
     if (ctx->elem_size != 4) bytes += (size_t)io_slots * stage;
     return bytes + sizeof(BulkShared) + 128;
 }
 
-int pick_stages(const dipaco_ctx *ctx, int units, int io_arrays, int io_slots)
+int pick_stages(const dipaco_ctx *ctx, int units, int io_arrays, int io_slots, bool shifted = true)
 {
     const size_t budget =
         std::min(SMEM_LIMIT, SMEM_PER_SM / (size_t)ctx->ctas_per_sm - 2 * SMEM_CTA_RESERVE);
     int best = 0;
     for (int s = 2; s <= BULK_MAX_STAGES; ++s)
-        if (bulk_smem_bytes(ctx, units, s, io_arrays, io_slots) <= budget) best = s;
+        if (bulk_smem_bytes(ctx, units, s, io_arrays, io_slots, shifted) <= budget) best = s;
     if (ctx->stages > 0) return ctx->stages <= best ? ctx->stages : best;
     return best;
 }
@@ -242,6 +245,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         rag_begin.push_back(b);
         rag_end.push_back(e);
     };
+    bool any_shifted = false;  // a bulk pass with a path buffer inside a 16-byte unit
     bool any_partial = false;
     for (const PassSpec &sp : specs)
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) any_partial = true;
@@ -269,8 +273,12 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (((sp.flags & PASS_CAST_IN) || sp.cast_out) && !ctx->cast_scratch) return DIPACO_ESTATE;
         bool aligned = ((uintptr_t)(theta + m.theta_off) % 16 == 0) &&
                        ((uintptr_t)(momentum + m.theta_off) % 16 == 0);
-        // the fp32 arrays all start at the same place within a 16-byte unit: a range can be cut
-        // so that every thread's first element is 16-byte aligned in all of them at once
+        // Can an element range be cut so that every tile (or thread) starts 16-byte aligned in
+        // all arrays that are not path buffers at once?  Ranges start where theta is 32-byte
+        // aligned, i.e. at elements k with (state_pos + k) % 8 == 0; the other fp32 arrays must
+        // then sit at the same place within a 16-byte unit as theta, and the cast scratch (path
+        // type) at the same element position within its unit.
+        const uintptr_t state_pos = ((uintptr_t)(theta + m.theta_off) % 32) / 4;  // in elements
         const uintptr_t state_rem = (uintptr_t)(theta + m.theta_off) % 16;
         bool state_congruent = (uintptr_t)(momentum + m.theta_off) % 16 == state_rem;
         if (ctx->optimizer == DIPACO_OPT_ADAM) {
@@ -281,6 +289,11 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (sp.flags & (PASS_PARTIAL_IN | PASS_PARTIAL_OUT)) {
             aligned = aligned && ((uintptr_t)(ctx->partial + m.partial_off) % 16 == 0);
             state_congruent = state_congruent && (uintptr_t)(ctx->partial + m.partial_off) % 16 == state_rem;
+        }
+        if ((sp.flags & PASS_CAST_IN) || sp.cast_out) {
+            const uintptr_t cast_addr = (uintptr_t)ctx->cast_scratch + (uintptr_t)m.cast_off * es;
+            aligned = aligned && cast_addr % 16 == 0;
+            state_congruent = state_congruent && cast_addr % 16 == (state_pos * es) % 16;
         }
         pd.contrib_begin = (int)contribs.size();
         for (size_t j = 0; j < sp.contributors.size(); ++j) {
@@ -310,13 +323,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
                 members.push_back(dst);
             }
         pd.member_count = (int)members.size() - pd.member_begin;
-        // destinations with the same position inside a 16-byte unit next to each other: the
-        // shifted vector kernel rebuilds its realigned units only when that position changes
-        // (the order of the destinations has no effect on the result)
-        if (!aligned)
-            std::stable_sort(members.begin() + pd.member_begin, members.end(), [](void *x, void *y) {
-                return ((uintptr_t)x & 15u) < ((uintptr_t)y & 15u);
-            });
+        pd.aligned_members = pd.member_count;
 
         // The vector kernel takes full tiles; the bulk-copy kernel also takes a partial last tile
         // as long as it is a whole number of 16-byte units of path data.
@@ -331,19 +338,40 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
         if (aligned && ctx->kernel == DIPACO_KERNEL_AUTO) full = (hi - lo) / unit * unit;
         bulk_begin[i] = lo; bulk_end[i] = lo + full;
         if (!aligned && state_congruent && ctx->kernel != DIPACO_KERNEL_SCALAR) {
-            // Path buffers at odd element offsets (or a range that starts inside a 16-byte unit):
-            // the shifted vector kernel takes whole steps from the first element at which theta
-            // is 16-byte aligned.  It reads the aligned 16-byte units around each thread's data,
-            // so the last 8 elements of the range stay with the one-element kernel: no load
-            // reaches past the module's slot in a path buffer.
-            const uintptr_t rem = (state_rem + (uintptr_t)(lo % 4) * 4) % 16;
-            const int64_t first = lo + (int64_t)((16 - rem) % 16) / 4;
-            const int64_t steps = hi - 8 > first ? (hi - 8 - first) / SHIFT_TILE : 0;
-            if (steps > 0) {
-                shv_begin[i] = first;
-                shv_end[i] = first + steps * SHIFT_TILE;
+            // Path buffers at odd element offsets (or a range that starts inside a 16-byte unit).
+            // The range of the vector or bulk-copy kernel starts at the first element at which
+            // theta is 32-byte aligned.  Both read the aligned 16-byte units around the data, so
+            // the last 8 elements of the range stay with the one-element kernel: no load reaches
+            // past the module's slot in a path buffer.
+            const int64_t first = lo + (int64_t)((8 - (state_pos + (uintptr_t)(lo % 8)) % 8) % 8);
+            int64_t covered = 0;
+            if (hi - 8 > first)
+                covered = ctx->kernel == DIPACO_KERNEL_VECTOR ? (hi - 8 - first) / SHIFT_TILE * SHIFT_TILE
+                                                              : (hi - 8 - first) / unit * unit;
+            if (covered > 0) {
+                // Destinations with the same position inside a 16-byte unit (at the range's
+                // tiles) next to each other, the aligned ones first: both kernels rebuild their
+                // realigned units only when that position changes, and the bulk-copy kernel
+                // writes the aligned ones with bulk stores.  The order has no effect on results.
+                const uintptr_t at_first = (uintptr_t)first * (uintptr_t)es;
+                auto shift_of = [at_first](void *x) { return ((uintptr_t)x + at_first) & 15u; };
+                std::stable_sort(members.begin() + pd.member_begin, members.end(),
+                                 [&](void *x, void *y) { return shift_of(x) < shift_of(y); });
+                int n_aligned = 0;
+                while (n_aligned < pd.member_count && shift_of(members[(size_t)(pd.member_begin + n_aligned)]) == 0)
+                    ++n_aligned;
+                pd.aligned_members = n_aligned;
+                if (ctx->kernel == DIPACO_KERNEL_VECTOR) {
+                    shv_begin[i] = first;
+                    shv_end[i] = first + covered;
+                    bulk_begin[i] = bulk_end[i] = lo;
+                } else {
+                    bulk_begin[i] = first;
+                    bulk_end[i] = first + covered;
+                    any_shifted = true;
+                }
                 add_ragged(i, lo, first);
-                add_ragged(i, shv_end[i], hi);
+                add_ragged(i, first + covered, hi);
                 continue;
             }
         }
@@ -418,6 +446,7 @@ int pack_launch(dipaco_ctx *ctx, const std::vector<PassSpec> &specs, const PtrLo
     out.io_arrays = io_arrays;
     out.units = units;
     out.aligned_kernel_is_vector = vector_kernel;
+    out.shifted = any_shifted;
     out.num_passes = (int)passes.size();
     out.total_items = (int)total_items;
     out.mean_contributors = bulk_elems > 0.0 ? contrib_elems / bulk_elems : 0.0;
@@ -473,23 +502,34 @@ int upload_blob(dipaco_ctx *ctx, const std::vector<unsigned char> &blob, cudaStr
     return DIPACO_OK;
 }
 
-template <typename PathT, int NU>
+template <typename PathT, int NU, bool SHIFTED>
 int launch_bulk_t(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages, int io_arrays, int io_slots,
-                  size_t smem, int attr_row, int attr_col, cudaStream_t stream)
+                  size_t smem, cudaStream_t stream)
 {
-    if (!ctx->smem_attr_set[attr_row][attr_col]) {
-        if (cudaFuncSetAttribute(sync_bulk_kernel<PathT, NU>,
+    bool &attr_set = ctx->smem_attr_set[sizeof(PathT) == 2 ? 1 : 0][NU == 1 ? 0 : (NU == 2 ? 1 : 2)][SHIFTED ? 1 : 0];
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(sync_bulk_kernel<PathT, NU, SHIFTED>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)SMEM_LIMIT) != cudaSuccess)
             return DIPACO_ECUDA;
-        ctx->smem_attr_set[attr_row][attr_col] = true;
+        attr_set = true;
     }
-    sync_bulk_kernel<PathT, NU><<<ctas, BULK_THREADS, smem, stream>>>(lp, stages, io_arrays, io_slots);
+    sync_bulk_kernel<PathT, NU, SHIFTED><<<ctas, SHIFTED ? BULK_SHIFTED_THREADS : BULK_THREADS, smem, stream>>>(
+        lp, stages, io_arrays, io_slots);
     return cudaGetLastError() == cudaSuccess ? DIPACO_OK : DIPACO_ECUDA;
 }
 
+template <typename PathT, bool SHIFTED>
+int launch_bulk_units(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int stages, int io_arrays,
+                      int io_slots, size_t smem, int nu, cudaStream_t stream)
+{
+    if (nu == 1) return launch_bulk_t<PathT, 1, SHIFTED>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, stream);
+    if (nu == 2) return launch_bulk_t<PathT, 2, SHIFTED>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, stream);
+    return launch_bulk_t<PathT, 4, SHIFTED>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, stream);
+}
+
 int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays, int nu,
-                double mean_contributors, cudaStream_t stream)
+                double mean_contributors, bool shifted, cudaStream_t stream)
 {
     // Shared memory is split between the ring of path tiles and the theta/momentum/result
     // buffers.  Launches dominated by many-contributor modules need the ring depth (10 stages
@@ -497,19 +537,15 @@ int launch_bulk(dipaco_ctx *ctx, const LaunchParams &lp, int ctas, int io_arrays
     const int wanted = ctx->stages > 0 ? std::min(ctx->stages, 10) : 10;
     const int min_stages = mean_contributors >= 8.0 ? wanted : std::min(wanted, 6);
     int io_slots = ctx->io_slots;
-    while (io_slots > 2 && pick_stages(ctx, nu, io_arrays, io_slots) < min_stages) --io_slots;
-    const int stages = pick_stages(ctx, nu, io_arrays, io_slots);
+    while (io_slots > 2 && pick_stages(ctx, nu, io_arrays, io_slots, shifted) < min_stages) --io_slots;
+    const int stages = pick_stages(ctx, nu, io_arrays, io_slots, shifted);
     if (stages < 2) return DIPACO_EINVAL;
-    const size_t smem = bulk_smem_bytes(ctx, nu, stages, io_arrays, io_slots);
-    const int col = nu == 1 ? 0 : (nu == 2 ? 1 : 2);
-    if (ctx->dtype == DIPACO_BF16) {
-        if (nu == 1) return launch_bulk_t<__nv_bfloat16, 1>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
-        if (nu == 2) return launch_bulk_t<__nv_bfloat16, 2>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
-        return launch_bulk_t<__nv_bfloat16, 4>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 1, col, stream);
-    }
-    if (nu == 1) return launch_bulk_t<float, 1>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 0, col, stream);
-    if (nu == 2) return launch_bulk_t<float, 2>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 0, col, stream);
-    return launch_bulk_t<float, 4>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, 0, col, stream);
+    const size_t smem = bulk_smem_bytes(ctx, nu, stages, io_arrays, io_slots, shifted);
+    if (ctx->dtype == DIPACO_BF16)
+        return shifted ? launch_bulk_units<__nv_bfloat16, true>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, nu, stream)
+                       : launch_bulk_units<__nv_bfloat16, false>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, nu, stream);
+    return shifted ? launch_bulk_units<float, true>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, nu, stream)
+                   : launch_bulk_units<float, false>(ctx, lp, ctas, stages, io_arrays, io_slots, smem, nu, stream);
 }
 
 int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *momentum,
@@ -555,7 +591,7 @@ int launch_packed(dipaco_ctx *ctx, const PackedLaunch &pl, float *theta, float *
                 sync_direct_kernel<float, 8><<<pl.bulk_ctas, 256, 0, stream>>>(lp);
             if (cudaGetLastError() != cudaSuccess) rc = DIPACO_ECUDA;
         } else {
-            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, pl.units, pl.mean_contributors, stream);
+            rc = launch_bulk(ctx, lp, pl.bulk_ctas, pl.io_arrays, pl.units, pl.mean_contributors, pl.shifted, stream);
         }
         if (rc != DIPACO_OK) return rc;
         ++ctx->launches;

@@ -34,6 +34,8 @@ struct PassDev {
     long long cast_off;     // elements into the cast scratch (valid with KPASS_CAST_IN)
     int contrib_begin, contrib_count;
     int member_begin, member_count;
+    int aligned_members;  // bulk-copy kernel: the first so many members are 16-byte aligned at the
+                          // pass's tiles (the host puts them first), the others sit inside a unit
     int flags;
     // dynamic scheduling of the bulk-copy kernel: this pass owns work items
     // [item_first, item_first + ceil(bulk_tiles / tiles_per_item)), each a run of full tiles
@@ -585,10 +587,11 @@ __device__ __forceinline__ void fence_proxy_async()
 constexpr int BULK_COMPUTE_WARPS = 8;
 constexpr int BULK_COMPUTE_THREADS = BULK_COMPUTE_WARPS * 32;
 constexpr int BULK_THREADS = BULK_COMPUTE_THREADS + 96;  // + load, store and scheduler warps
+constexpr int BULK_SHIFTED_STORE_WARPS = 4;  // the variant for shifted path buffers stores with four warps
+constexpr int BULK_SHIFTED_THREADS = BULK_THREADS + 32 * (BULK_SHIFTED_STORE_WARPS - 1);
 constexpr int BULK_MAX_STAGES = 32;
 constexpr int BULK_SCHED_DEPTH = 4;
 constexpr int BULK_MAX_IO_SLOTS = 4;  // buffers of theta/momentum/partial/result tiles
-constexpr int BULK_ITEM_READERS = BULK_COMPUTE_WARPS + 2;  // warps that consume every work item
 constexpr unsigned long long BULK_WAIT_LIMIT_NS = 4000000000ull;  // every wait gives up after 4 s
 
 // Bounded wait: returns false (and records the failure) if the phase does not complete in time.
@@ -615,10 +618,13 @@ struct BulkShared {
     uint64_t io_empty[BULK_MAX_IO_SLOTS];   // result tiles drained by the store warp
     uint64_t out_ready[BULK_MAX_IO_SLOTS];  // compute warps finished writing the result tiles
     uint64_t sched_full[BULK_SCHED_DEPTH];   // a work item was published by the scheduler warp
-    uint64_t sched_empty[BULK_SCHED_DEPTH];  // all ten consumer warps have read it
+    uint64_t sched_empty[BULK_SCHED_DEPTH];  // all consumer warps (compute, load, store) have read it
     long long sched_begin[BULK_SCHED_DEPTH], sched_end[BULK_SCHED_DEPTH];
     int sched_pass[BULK_SCHED_DEPTH];        // -1 = no more work
     float slot_coeff[BULK_MAX_STAGES];
+    unsigned slot_shift[BULK_MAX_STAGES];  // bytes from the start of a ring slot to the tile's data
+    // store warps: the destinations that share the current shift (one list per warp)
+    unsigned long long store_dst[BULK_SHIFTED_STORE_WARPS][32];
     const void *batch_src[32];
     float batch_coeff[32];
 };
@@ -684,21 +690,33 @@ struct ItemWalk {
 };
 
 // NU = 16-byte units of path data per compute thread and tile; tile = 256 * NU * UE elements.
-template <typename PathT, int NU>
-__global__ void __launch_bounds__(BULK_THREADS, 1)
+// SHIFTED: the tiles of theta, momentum, partial sums, second moment and cast scratch are 16-byte
+// aligned as always (the host cuts the range that way), but a path buffer may sit at any element
+// alignment, each its own.  A contributor's tile is then loaded from the aligned address at or
+// before it (16 bytes more) and the compute warps cut their bytes out of two neighbouring units;
+// a member that is not aligned is written by the store warp itself, in aligned 16-byte units put
+// together from the cast tile, instead of by a bulk store.
+template <typename PathT, int NU, bool SHIFTED = false>
+__global__ void __launch_bounds__(SHIFTED ? BULK_SHIFTED_THREADS : BULK_THREADS, 1)
 sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
 {
+    // warps: 0..7 compute, 8 load, 9.. store (one, or four in the shifted variant), then the scheduler
+    constexpr int STORE_WARPS = SHIFTED ? BULK_SHIFTED_STORE_WARPS : 1;
+    constexpr int FIRST_STORE_WARP = BULK_COMPUTE_WARPS + 1;
+    constexpr int SCHED_WARP = FIRST_STORE_WARP + STORE_WARPS;
+    constexpr int ITEM_READERS = BULK_COMPUTE_WARPS + 1 + STORE_WARPS;  // warps that consume every work item
     constexpr int UE = Unit<PathT>::UE;
     constexpr int EPT = UE * NU;                         // elements per compute thread
     constexpr int TILE = BULK_COMPUTE_THREADS * EPT;     // elements per tile
     constexpr unsigned STAGE_BYTES = TILE * sizeof(PathT);
+    constexpr unsigned STAGE_STRIDE = STAGE_BYTES + (SHIFTED ? 16u : 0u);  // ring slot size
     constexpr unsigned F32_TILE_BYTES = TILE * 4u;
     constexpr bool NEED_CAST_TILE = sizeof(PathT) != 4;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // layout: ring | io[io_slots][io_arrays] fp32 tiles | cast tile[io_slots] (bf16 only) | BulkShared
     unsigned char *ring = smem_raw;
-    unsigned char *io = ring + (size_t)stages * STAGE_BYTES;
+    unsigned char *io = ring + (size_t)stages * STAGE_STRIDE;
     unsigned char *cast_tiles = io + (size_t)io_slots * io_arrays * F32_TILE_BYTES;
     BulkShared *sh = reinterpret_cast<BulkShared *>(
         cast_tiles + (NEED_CAST_TILE ? (size_t)io_slots * STAGE_BYTES : (size_t)0));
@@ -713,11 +731,11 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
         }
         for (int d = 0; d < BULK_SCHED_DEPTH; ++d) {
             ptx::mbar_init(&sh->sched_full[d], 1);
-            ptx::mbar_init(&sh->sched_empty[d], BULK_ITEM_READERS);
+            ptx::mbar_init(&sh->sched_empty[d], ITEM_READERS);
         }
         for (int b = 0; b < io_slots; ++b) {
             ptx::mbar_init(&sh->io_full[b], 1);
-            ptx::mbar_init(&sh->io_empty[b], 1);
+            ptx::mbar_init(&sh->io_empty[b], STORE_WARPS);
             ptx::mbar_init(&sh->out_ready[b], BULK_COMPUTE_WARPS);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -741,7 +759,7 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
     RingPos io_pos;  // theta/momentum/result buffer of the current tile (advances once per tile)
     RingPos q;       // ring position of this role
 
-    if (warp == BULK_COMPUTE_WARPS + 2) {
+    if (warp == SCHED_WARP) {
         // ------------------------------------------------------------------ scheduler warp
         if (lane == 0) {
             int slot = 0;
@@ -842,11 +860,19 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                         ok = bounded_wait(&sh->empty[s], q.phase ^ 1u, p.error_word, 2);
                         if (!ok) break;
                         sh->slot_coeff[s] = sh->batch_coeff[u];
-                        const unsigned path_bytes = n * (unsigned)sizeof(PathT);
+                        unsigned path_bytes = n * (unsigned)sizeof(PathT);
+                        const PathT *from = static_cast<const PathT *>(sh->batch_src[u]) + k0;
+                        if constexpr (SHIFTED) {
+                            // start at the aligned address at or before the tile; the bytes in
+                            // front of the data and the 16 more behind it lie in the same aligned
+                            // units as the data
+                            const unsigned shift = (unsigned)(reinterpret_cast<uintptr_t>(from) & 15u);
+                            sh->slot_shift[s] = shift;
+                            from = reinterpret_cast<const PathT *>(reinterpret_cast<const char *>(from) - shift);
+                            if (shift) path_bytes += 16u;
+                        }
                         ptx::mbar_arrive_expect_tx(&sh->full[s], path_bytes);
-                        ptx::bulk_load(ring + (size_t)s * STAGE_BYTES,
-                                       static_cast<const PathT *>(sh->batch_src[u]) + k0, path_bytes,
-                                       &sh->full[s]);
+                        ptx::bulk_load(ring + (size_t)s * STAGE_STRIDE, from, path_bytes, &sh->full[s]);
                         q.advance(stages);
                     }
                 }
@@ -867,15 +893,18 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                 bounded_wait(&sh->io_full[io_pos.slot], io_pos.phase, p.error_word, 3);
             }
         }
-    } else if (warp == BULK_COMPUTE_WARPS + 1) {
-        // ------------------------------------------------------------------ store warp
+    } else if (warp >= FIRST_STORE_WARP && warp < SCHED_WARP) {
+        // ------------------------------------------------------------------ store warp(s)
+        // The first store warp issues every bulk store; in the shifted variant all of them share
+        // the members that are written with ordinary stores.
+        const int rank = warp - FIRST_STORE_WARP;
         bool ok = true;
         while (ok && walk.next(k0, n, ok)) {
             const PassDev pass = p.passes[walk.pass];
             const int b = io_pos.slot;
             ok = bounded_wait(&sh->out_ready[b], io_pos.phase, p.error_word, 4);
             if (!ok) break;
-            if (lane == 0) {
+            if (lane == 0 && rank == 0) {
                 if (pass.flags & KPASS_UPDATE) {
                     ptx::bulk_store(p.theta + pass.theta_off + k0, io_tile(b, 0), n * 4u);
                     ptx::bulk_store(p.momentum + pass.theta_off + k0, io_tile(b, 1), n * 4u);
@@ -887,9 +916,60 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                     ptx::bulk_store(p.partial + pass.partial_off + k0, io_tile(b, 2), n * 4u);
             }
             const unsigned char *src = cast_tile(b);
-            for (int j = lane; j < pass.member_count; j += 32) {
+            const int bulk_members = rank != 0 ? 0 : (SHIFTED ? pass.aligned_members : pass.member_count);
+            for (int j = lane; j < bulk_members; j += 32) {
                 PathT *dst = static_cast<PathT *>(p.members[pass.member_begin + j]) + k0;
                 ptx::bulk_store(dst, src, n * (unsigned)sizeof(PathT));
+            }
+            if constexpr (SHIFTED) {
+                // Members inside a 16-byte unit (the host puts them after the aligned ones, sorted
+                // by their shift).  Thirty-two at a time, one per lane; for every shift among them
+                // the store warps walk the tile once between them, build each aligned 16-byte unit
+                // of output from two neighbouring units of the cast tile and store it to all
+                // members with that shift.  The bytes in front of a member's first aligned unit
+                // and behind its last one go out element by element (first store warp).
+                const uint4 *tile16 = reinterpret_cast<const uint4 *>(src);
+                const PathT *tile_el = reinterpret_cast<const PathT *>(src);
+                const int units = (int)(n * (unsigned)sizeof(PathT) / 16u);
+                constexpr int PER = 16 / (int)sizeof(PathT);
+                for (int base = pass.aligned_members; base < pass.member_count; base += 32) {
+                    const bool valid = base + lane < pass.member_count;
+                    char *mine = valid ? reinterpret_cast<char *>(static_cast<PathT *>(
+                                             p.members[pass.member_begin + base + lane]) + k0)
+                                       : nullptr;
+                    const unsigned my_shift = (unsigned)(reinterpret_cast<uintptr_t>(mine) & 15u);
+                    unsigned todo = __ballot_sync(0xffffffffu, valid);
+                    while (todo) {
+                        const int leader = __ffs(todo) - 1;
+                        const unsigned shift = __shfl_sync(0xffffffffu, my_shift, leader);
+                        const unsigned group = __ballot_sync(0xffffffffu, valid && my_shift == shift) & todo;
+                        todo &= ~group;
+                        // the group's first aligned units, side by side in shared memory
+                        __syncwarp();
+                        if ((group >> lane) & 1u)
+                            sh->store_dst[rank][__popc(group & ((1u << lane) - 1u))] =
+                                (unsigned long long)reinterpret_cast<uintptr_t>(mine) + 16u - shift;
+                        __syncwarp();
+                        const int count = __popc(group);
+                        // aligned unit i of the output holds tile bytes [16 i + 16 - shift, 16 i + 32 - shift)
+                        for (int i = rank * 32 + lane; i + 1 < units; i += 32 * STORE_WARPS) {
+                            const uint4 unit = cut16(tile16[i], tile16[i + 1], 16u - shift);
+#pragma unroll 4
+                            for (int m = 0; m < count; ++m)
+                                __stcs(reinterpret_cast<uint4 *>(sh->store_dst[rank][m]) + i, unit);
+                        }
+                    }
+                    // edges: each lane for its own member
+                    if (valid && rank == 0) {
+                        PathT *dst = reinterpret_cast<PathT *>(mine);
+                        const int head = (int)(16u - my_shift) / (int)sizeof(PathT);
+#pragma unroll
+                        for (int e = 0; e < PER; ++e) {
+                            const unsigned at = e < head ? (unsigned)e : n - (unsigned)PER + (unsigned)e;
+                            dst[at] = tile_el[at];
+                        }
+                    }
+                }
             }
             ptx::bulk_commit();
             ptx::bulk_wait_read_all();
@@ -948,10 +1028,18 @@ sync_bulk_kernel(LaunchParams p, int stages, int io_arrays, int io_slots)
                 ok = bounded_wait(&sh->full[s], q.phase, p.error_word, 6);
                 if (!ok) break;
                 const float c = sh->slot_coeff[s];
-                const uint4 *slot = reinterpret_cast<const uint4 *>(ring + (size_t)s * STAGE_BYTES);
+                const uint4 *slot = reinterpret_cast<const uint4 *>(ring + (size_t)s * STAGE_STRIDE);
                 uint4 raw[NU];
 #pragma unroll
                 for (int u = 0; u < NU; ++u) raw[u] = slot[u * BULK_COMPUTE_THREADS + ct];
+                if constexpr (SHIFTED) {
+                    const unsigned shift = sh->slot_shift[s];
+                    if (shift) {  // the same for the whole CTA
+#pragma unroll
+                        for (int u = 0; u < NU; ++u)
+                            raw[u] = cut16(raw[u], slot[u * BULK_COMPUTE_THREADS + ct + 1], shift);
+                    }
+                }
 #pragma unroll
                 for (int u = 0; u < NU; ++u) {
                     float x[UE];

@@ -121,16 +121,17 @@ inline bool build_grid(Grid &g, int L, const int32_t *K, const int64_t *N, int P
     g.scratch_elems = 0;
     g.cast_elems = 0;
     for (auto &m : g.modules) {
-        m.cast_off = g.cast_elems;
-        g.cast_elems += (m.numel + 7) / 8 * 8;
+        // A module's slot in either scratch starts where its theta starts within a group of eight
+        // elements (at a multiple of eight when theta_off is one): an element range cut so that
+        // theta is 32-byte aligned is then 16-byte aligned in the partial sums (fp32) and in the
+        // cast scratch (path type) too.
+        m.cast_off = g.cast_elems + (m.theta_off & 7);
+        g.cast_elems = (m.cast_off + m.numel + 7) / 8 * 8;
         m.partial_off = -1;
         if (g.num_chunks > 1 && !m.members.empty() &&
             g.chunk_of(m.members.front()) != g.chunk_of(m.members.back())) {
-            // A module's slab starts where its theta starts within a 16-byte unit (at a multiple
-            // of four elements when theta_off is one), so that vector and bulk accesses that are
-            // aligned for theta are aligned for the partial sum too.
-            m.partial_off = g.scratch_elems + (m.theta_off & 3);
-            g.scratch_elems = (m.partial_off + m.numel + 3) / 4 * 4;
+            m.partial_off = g.scratch_elems + (m.theta_off & 7);
+            g.scratch_elems = (m.partial_off + m.numel + 7) / 8 * 8;
         }
     }
     return true;

@@ -245,7 +245,7 @@ def test_masked_paths_are_not_read_and_nan_propagates():
     assert torch.isnan(state[0]).sum().item() == 1
 
 
-def test_misaligned_path_pointers_on_small_modules_take_the_scalar_path():
+def test_misaligned_path_pointers_on_small_modules():
     cfg = synth.SyncConfig("mis", (1, 2, 2), (4100, 2052, 1000), "bf16", seed=9)
     pr = synth.make_problem(cfg, DEV)
     before = host_state(clone_problem(pr))
@@ -263,12 +263,13 @@ def test_misaligned_path_pointers_on_small_modules_take_the_scalar_path():
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("chunk", [0, 4])
-def test_path_buffers_at_any_element_alignment_take_the_shifted_vector_kernel(dtype, chunk):
+def test_path_buffers_at_any_element_alignment(dtype, chunk):
     """Every path copy starts at its own element offset within a 16-byte unit (all eight of them
     for bf16, all four for fp32) and the level sizes are odd, so the modules of theta, the slots
-    inside the copies and the partial sums all start inside 16-byte units.  The vector kernel for
-    shifted buffers takes the bulk of every module, the one-element kernel a few elements before
-    and after: against the oracle, and bitwise equal to the one-element kernel on its own."""
+    inside the copies and the partial sums all start inside 16-byte units.  The bulk-copy kernel
+    (default) or the vector kernel, each in its variant for shifted buffers, takes the bulk of
+    every module, the one-element kernel a few elements before and after: against the oracle,
+    and bitwise equal to the one-element kernel on its own."""
     cfg = synth.SyncConfig("shifted", (1, 3, 3), (3 * 2048 + 5, 2 * 2048 + 1003, 5 * 2048 + 77), dtype,
                            weights="tokens", momentum_std=1e-4, seed=9)
     pr = synth.make_problem(cfg, DEV)

@@ -171,8 +171,16 @@ def test_chunk_count_and_scratch_size():
     cfg = synth.CONFIGS["grid16x16"].scaled((1000, 1001, 1002))
     ctx = plan_ctx(cfg, chunk_paths=32)
     n, scratch = B.dipaco_plan_chunks(ctx)
-    # shared level and the 16 level-2 modules span chunks; level-1 modules live inside one chunk
-    assert n == 8 and scratch == 1000 + 16 * 1004
+    # shared level and the 16 level-2 modules span chunks; level-1 modules live inside one chunk.
+    # A module's slot starts where its theta starts within a group of eight elements and slots
+    # do not share such a group: at most 14 elements of padding per module.
+    need = 1000 + 16 * 1002
+    assert n == 8 and need <= scratch <= need + 17 * 14 and scratch % 8 == 0
+    B.dipaco_destroy(ctx)
+    # sizes that are multiples of eight need no padding at all
+    even = synth.CONFIGS["grid16x16"].scaled((1000, 1008, 1016))
+    ctx = plan_ctx(even, chunk_paths=32)
+    assert B.dipaco_plan_chunks(ctx) == (8, 1000 + 16 * 1016)
     B.dipaco_destroy(ctx)
     ctx = plan_ctx(cfg, chunk_paths=0)
     assert B.dipaco_plan_chunks(ctx) == (1, 0)
