@@ -71,10 +71,21 @@ enum {
 
 /* kernel selection for dipaco_set_kernel */
 enum {
-    DIPACO_KERNEL_AUTO = 0,   /* bulk-copy (TMA) pipeline for 16-byte aligned full tiles, scalar rest */
-    DIPACO_KERNEL_VECTOR = 1, /* 128-bit register loads/stores for aligned full tiles, scalar rest    */
-    DIPACO_KERNEL_SCALAR = 2  /* one element per thread everywhere (any alignment)                    */
+    DIPACO_KERNEL_AUTO = 0,   /* bulk-copy (TMA) pipeline, one element per thread for the few elements
+                                 before and after its range                                            */
+    DIPACO_KERNEL_VECTOR = 1, /* 128-bit register loads/stores on whole steps, one element per thread
+                                 for the rest                                                         */
+    DIPACO_KERNEL_SCALAR = 2  /* one element per thread everywhere                                    */
 };
+/*
+ * Alignment.  Nothing has to be aligned beyond its element size.  Path copies may start at any
+ * element boundary, each at its own, and level sizes may be odd (modules and slots then start
+ * inside 16-byte units): the bulk-copy and the vector kernel each have a variant that loads the
+ * aligned 16-byte units around the data and writes realigned units, at 0.91-0.95 of the speed of
+ * fully aligned buffers (bulk-copy kernel).  They need theta, momentum (and the second moment) to
+ * sit at the same place within a 16-byte unit, which holds whenever these arrays are allocated the
+ * same way; otherwise the module falls back to one element per thread.
+ */
 
 /*
  * Build a context for one module grid (Algorithm 1, "Require" lines; Section 2.2 notation).
