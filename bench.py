@@ -39,7 +39,7 @@ REF_SAMPLE_NUMEL = 1_000_000      # parameters per level per step in the referen
 # digest is checked and "traffic" is null after any change to them.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.9919
 NCU_CAPTURE_SOURCES = ("kernels.cuh", "dipaco.cu", "plan.hpp")
-NCU_CAPTURE_SOURCES_SHA256 = "8556fee352be290cd0cac9acb70132f55b758231eff625b706abd6f55a4626b6"
+NCU_CAPTURE_SOURCES_SHA256 = "63fd72cb32bba49c5bfc6f80f7e446524e0064dc8ead76279df492ad99f8e61d"
 NCU_CAPTURE_COMMAND = ("ncu --set full --clock-control none -k regex:sync_bulk_kernel -s 3 -c 3 "
                        "python bench.py --level-numel 2000000 --steps 3 --warmup 3 --no-e2e "
                        "--no-chunked --no-cpu-baseline --no-variants --no-other-workloads")

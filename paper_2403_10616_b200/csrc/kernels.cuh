@@ -12,6 +12,10 @@
 //                                 ring with bulk async copies (TMA, 1-D), eight warps reduce and
 //                                 apply the optimiser step, one warp scatters the result tile to
 //                                 every path with bulk stores from shared memory.
+//   sync_bulk_kernel<PathT,NU,true>  the same for path buffers at any element alignment: tiles
+//                                 loaded from the aligned address at or before them and cut out
+//                                 of neighbouring 16-byte units; shifted destinations written in
+//                                 realigned units by four store warps.
 #pragma once
 
 #include <cuda_bf16.h>
