@@ -585,7 +585,7 @@ def run_other_workloads(args, skip_name, tune, local, peak):
     # the last entry is the 16x16 grid with an odd level size: every module of theta and every slot
     # of every path copy then starts inside a 16-byte unit (rows of one block: all eight positions),
     # so the bulk-copy kernel cannot take it and the shifted vector kernel does
-    odd = synth.CONFIGS["grid16x16"].scaled((20_000_003,) * 3, name="grid16x16-odd-level-size")
+    odd = synth.CONFIGS["grid16x16-odd-level-size"]
     for name in ("grid2x2", "grid4x4", "grid16x16-masked", "grid4x4x4x4", odd.name):
         if name == skip_name:
             continue

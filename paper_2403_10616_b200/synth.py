@@ -81,6 +81,11 @@ CONFIGS = {
                                    weights="zipf", mask_prob=0.2, chunk_paths=32),
     "grid4x4x4x4": SyncConfig("grid4x4x4x4", (1, 4, 4, 4, 4), (20_000_000,) + (10_000_000,) * 4,
                               "bf16", outlier_frac=0.01),
+    # the 16x16 grid with an odd level size: every module of theta after the first and every slot
+    # of a path copy starts inside a 16-byte unit, and copies that are rows of one block sit at all
+    # eight positions within a unit
+    "grid16x16-odd-level-size": SyncConfig("grid16x16-odd-level-size", (1, 16, 16), (20_000_003,) * 3,
+                                           "bf16", chunk_paths=32),
 }
 
 

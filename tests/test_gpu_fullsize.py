@@ -1,8 +1,9 @@
 """Parity at the benchmark's full sizes, in the launch configurations bench.py times.
 
 Workloads: the 16x16 grid (256 paths, 150M parameters per path, bf16), the same with 20 % of the
-paths not reporting and Zipf weights, and the 4x4x4x4 grid (256 paths, 60M parameters per path,
-1 % of the deltas a hundred times larger).  Legs: resident one-pass (default kernel and tuning),
+paths not reporting and Zipf weights, the 4x4x4x4 grid (256 paths, 60M parameters per path,
+1 % of the deltas a hundred times larger), and the 16x16 grid with an odd level size (20,000,003:
+modules and slots inside 16-byte units, the kernel variant for shifted buffers).  Legs: resident one-pass (default kernel and tuning),
 the chunk walk (chunks of 32 paths) and the host-buffer entry point.
 
 The oracle cannot run 38.4e9 path elements in test time; elements are independent, so it is
@@ -121,7 +122,7 @@ def assert_every_copy_is_the_cast_of_its_module(problem):
                     assert torch.equal(slot, want)
 
 
-@pytest.mark.parametrize("name", ["grid16x16", "grid16x16-masked", "grid4x4x4x4"])
+@pytest.mark.parametrize("name", ["grid16x16", "grid16x16-masked", "grid4x4x4x4", "grid16x16-odd-level-size"])
 def test_full_size_sampled_parity_properties_and_reproducibility(name):
     cfg = synth.CONFIGS[name]
     need = cfg.path_params * 2 + 8 * cfg.module_params
